@@ -1,0 +1,198 @@
+"""CPU oracle of the quantized selective-state-update decode step -- TEST INFRASTRUCTURE ONLY.
+
+A thin ctypes wrapper over ``ssdq_oracle.cpp`` (plain C++17, compiled on first use with g++).
+Nothing in the product package imports this module; it serves the tests, the smoke check and the
+CPU-baseline leg of the benchmark.  It shares no code with the CUDA path.
+
+Every function mirrors one exported symbol of the C++ file; see that file for the passages of the
+paper each step follows (Eq. 1, Eq. 2, Appendix B "Formats" and "Dithers").
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import numpy as np
+
+FP16, BF16, E4M3, FP32 = 0, 1, 2, 3
+RTN, SR, WEYL = 0, 1, 2
+FORMAT_NAMES = {FP16: "fp16", BF16: "bf16", E4M3: "e4m3", FP32: "fp32"}
+RULE_NAMES = {RTN: "rtn", SR: "sr", WEYL: "weyl"}
+CODE_DTYPE = {FP16: np.uint16, BF16: np.uint16, E4M3: np.uint8, FP32: np.uint32}
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "ssdq_oracle.cpp")
+_LIB = os.path.join(_HERE, "libssdq_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle (g++, no fast-math, no FMA contraction).  Returns the library path."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["g++", "-O2", "-std=c++17", "-ffp-contract=off", "-fopenmp", "-shared", "-fPIC",
+               "-o", _LIB, _SRC]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(build())
+        u32, u64, f32, i32 = ctypes.c_uint32, ctypes.c_uint64, ctypes.c_float, ctypes.c_int
+        vp = ctypes.c_void_p
+        L.oracle_weyl_acc.restype = u32
+        L.oracle_weyl_acc.argtypes = [u32] * 5
+        L.oracle_philox4x32_10.restype = None
+        L.oracle_philox4x32_10.argtypes = [vp, vp, vp]
+        L.oracle_exp_spec.restype = f32
+        L.oracle_exp_spec.argtypes = [f32]
+        L.oracle_round.restype = f32
+        L.oracle_round.argtypes = [f32, i32, i32, u32]
+        L.oracle_encode.restype = u32
+        L.oracle_encode.argtypes = [f32, i32]
+        L.oracle_decode.restype = f32
+        L.oracle_decode.argtypes = [u32, i32]
+        L.oracle_threshold.restype = u32
+        L.oracle_threshold.argtypes = [i32, u32, u32, u32, u64, u64, u32]
+        L.oracle_round_array.restype = None
+        L.oracle_round_array.argtypes = [vp, vp, u64, i32, i32, vp]
+        L.oracle_exp_spec_array.restype = None
+        L.oracle_exp_spec_array.argtypes = [vp, u64, vp]
+        L.oracle_state_update.restype = i32
+        L.oracle_state_update.argtypes = [vp, vp, i32, u32, u32, u32, u32, u32, vp, vp, vp, i32, vp, vp, vp, vp,
+                                          i32, u32, u32, u32, u64, u32, u32]
+        L.oracle_quantize_store.restype = i32
+        L.oracle_quantize_store.argtypes = [vp, vp, vp, u64, u32, i32, u32, i32, u32, u32, u32, u64, u64, u32]
+        L.oracle_dequantize.restype = None
+        L.oracle_dequantize.argtypes = [vp, vp, u64, i32, u32, vp]
+        L.oracle_num_threads.restype = i32
+        L.oracle_num_threads.argtypes = []
+        _lib = L
+    return _lib
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _f32(a):
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    return a
+
+
+# ---- elementary functions -------------------------------------------------------------------
+def weyl_acc(r, c, layer, seed, t) -> int:
+    m = 0xFFFFFFFF
+    return lib().oracle_weyl_acc(r & m, c & m, layer & m, seed & m, t & m)
+
+
+def weyl_u24(r, c, layer, seed, t) -> int:
+    return weyl_acc(r, c, layer, seed, t) >> 8
+
+
+def philox4x32_10(ctr, key):
+    c = np.asarray(ctr, dtype=np.uint32).copy()
+    k = np.asarray(key, dtype=np.uint32).copy()
+    out = np.zeros(4, dtype=np.uint32)
+    lib().oracle_philox4x32_10(_ptr(c), _ptr(k), _ptr(out))
+    return out
+
+
+def exp_spec(z):
+    z = _f32(np.atleast_1d(z))
+    out = np.empty_like(z)
+    lib().oracle_exp_spec_array(_ptr(z), z.size, _ptr(out))
+    return out
+
+
+def threshold(rule, flat, t, layer=0, weyl_seed=0, weyl_block=16, sr_seed=0) -> int:
+    return lib().oracle_threshold(rule, layer, weyl_seed, weyl_block, sr_seed, flat, t & 0xFFFFFFFF)
+
+
+def thresholds(rule, flats, t, layer=0, weyl_seed=0, weyl_block=16, sr_seed=0):
+    return np.array([threshold(rule, int(f), t, layer, weyl_seed, weyl_block, sr_seed) for f in flats],
+                    dtype=np.uint32)
+
+
+def round_values(v, U, fmt, rule):
+    """Eq. 2 on the local grid of `fmt`, elementwise; returns the rounded values as float32."""
+    v = _f32(np.atleast_1d(v))
+    U = np.ascontiguousarray(np.broadcast_to(np.asarray(U, dtype=np.uint32), v.shape))
+    out = np.empty_like(v)
+    lib().oracle_round_array(_ptr(v), _ptr(U), v.size, fmt, rule, _ptr(out))
+    return out
+
+
+def encode(q, fmt):
+    q = _f32(np.atleast_1d(q))
+    return np.array([lib().oracle_encode(float(x), fmt) for x in q.ravel()],
+                    dtype=CODE_DTYPE[fmt]).reshape(q.shape)
+
+
+def decode(codes, fmt):
+    codes = np.atleast_1d(codes)
+    return np.array([lib().oracle_decode(int(c), fmt) for c in codes.ravel()],
+                    dtype=np.float32).reshape(codes.shape)
+
+
+# ---- the decode step ------------------------------------------------------------------------
+def state_update(state, scales, fmt, scale_block, x, dt, A, Bm, Cm, D, rule, step_t, *, layer=0,
+                 weyl_seed=0, weyl_block=16, sr_seed=0, batch_index_base=0):
+    """One decode step of one layer, in place on `state` (and `scales`).  Returns y [B,H,P] float32.
+
+    state [B,H,P,N] of CODE_DTYPE[fmt] (float32 viewed as uint32 for FP32); x [B,H,P]; dt [B,H];
+    A [H] or [H,N]; Bm, Cm [B,N]; D [H] or None.
+    """
+    Bsz, H, P, N = state.shape
+    assert state.flags.c_contiguous and state.dtype == CODE_DTYPE[fmt]
+    x, dt, A, Bm, Cm = _f32(x), _f32(dt), _f32(A), _f32(Bm), _f32(Cm)
+    D = None if D is None else _f32(D)
+    assert x.shape == (Bsz, H, P) and dt.shape == (Bsz, H) and Bm.shape == (Bsz, N) and Cm.shape == (Bsz, N)
+    a_per_state = int(A.ndim == 2)
+    assert A.shape == ((H, N) if a_per_state else (H,))
+    y = np.empty((Bsz, H, P), dtype=np.float32)
+    if scales is not None:
+        assert scales.dtype == np.float32 and scales.flags.c_contiguous
+    rc = lib().oracle_state_update(_ptr(state), _ptr(scales), fmt, scale_block, Bsz, H, P, N, _ptr(x), _ptr(dt),
+                                   _ptr(A), a_per_state, _ptr(Bm), _ptr(Cm), _ptr(D), _ptr(y), rule, layer,
+                                   weyl_seed, weyl_block, sr_seed, batch_index_base, step_t)
+    if rc != 0:
+        raise ValueError("oracle_state_update: undefined argument combination")
+    return y
+
+
+def quantize_store(src, fmt, rule, step_t, *, scale_block=0, layer=0, weyl_seed=0, weyl_block=16, sr_seed=0,
+                   row_index_base=0):
+    """Quantise float32 `src` [n_rows, row_len]; returns (codes, scales or None)."""
+    src = _f32(src)
+    n_rows, row_len = src.shape
+    codes = np.zeros((n_rows, row_len), dtype=CODE_DTYPE[fmt])
+    scales = np.zeros((n_rows, row_len // scale_block), dtype=np.float32) if fmt == E4M3 else None
+    rc = lib().oracle_quantize_store(_ptr(src), _ptr(codes), _ptr(scales), n_rows, row_len, fmt, scale_block, rule,
+                                     layer, weyl_seed, weyl_block, sr_seed, row_index_base, step_t)
+    if rc != 0:
+        raise ValueError("oracle_quantize_store: undefined argument combination")
+    return codes, scales
+
+
+def dequantize(codes, scales, fmt, scale_block=0):
+    codes = np.ascontiguousarray(codes)
+    out = np.empty(codes.shape, dtype=np.float32)
+    lib().oracle_dequantize(_ptr(codes), _ptr(scales), codes.size, fmt, max(scale_block, 1), _ptr(out))
+    return out
+
+
+def new_state(shape, fmt, scale_block=0):
+    """All-zero state (h_0 = 0) and its scale array (E4M3: scale of an all-zero block)."""
+    Bsz, H, P, N = shape
+    state = np.zeros(shape, dtype=CODE_DTYPE[fmt])
+    scales = None
+    if fmt == E4M3:
+        n_scales = Bsz * H if scale_block == P * N and scale_block != N else Bsz * H * P * (N // scale_block)
+        scales = np.full(n_scales, np.finfo(np.float32).tiny, dtype=np.float32)
+    return state, scales
+
+
+def num_threads() -> int:
+    return lib().oracle_num_threads()

@@ -1,0 +1,247 @@
+"""Pins of the oracle's decode step: exp_spec, Proposition 1 as an end-to-end identity, Lemma 1,
+the closed form of Eq. 1 without rounding, scale invariance of the E4M3 store, and an independent
+brute-force restatement on tiny states."""
+from fractions import Fraction
+import math
+
+import numpy as np
+import pytest
+
+import oracle
+from oracle import FP16, BF16, E4M3, FP32, RTN, SR, WEYL
+from paper_2609_39185_b200 import workloads
+
+
+# ---- exp_spec ------------------------------------------------------------------------------
+def test_exp_spec_accuracy_and_fixed_points():
+    assert oracle.exp_spec(0.0)[0] == 1.0 and oracle.exp_spec(-0.0)[0] == 1.0
+    rng = np.random.default_rng(0)
+    z = np.concatenate([-87.0 * rng.random(400000), -10.0 ** rng.uniform(-8, 0, 100000),
+                        np.array([-87.0, -1e-45, -100.0, -1e30])]).astype(np.float32)
+    got = oracle.exp_spec(z).astype(np.float64)
+    want = np.exp(np.maximum(z.astype(np.float64), -87.0))
+    ulp = np.spacing(want.astype(np.float32)).astype(np.float64)
+    assert np.max(np.abs(got - want) / ulp) <= 2.0
+    assert np.all(got >= np.finfo(np.float32).tiny)                 # always a normal number
+    assert np.all(got <= 1.0)                                       # a decay never exceeds one
+    zs = np.sort(z)
+    assert np.all(np.diff(oracle.exp_spec(zs)) >= -np.spacing(oracle.exp_spec(zs))[1:] * 2)
+
+
+# ---- Proposition 1 on the real update --------------------------------------------------------
+def run_scalar_recurrence(w_over_step, h0, T, rule, fmt=FP16):
+    """N = 16 independent entries with a = 1 (A = 0), dt = x = 1 and B[n] = w[n]: h <- Q(h + w)."""
+    N = len(w_over_step)
+    step = 2.0**-10
+    state = oracle.encode(np.full((1, 1, 1, N), h0, dtype=np.float32), fmt).reshape(1, 1, 1, N)
+    A = np.zeros(1, np.float32)
+    x = np.ones((1, 1, 1), np.float32)
+    dt = np.ones((1, 1), np.float32)
+    Bm = (np.asarray(w_over_step, dtype=np.float64) * step).astype(np.float32).reshape(1, N)
+    Cm = np.zeros((1, N), np.float32)
+    for t in range(1, T + 1):
+        oracle.state_update(state, None, fmt, 0, x, dt, A, Bm, Cm, None, rule, t, weyl_block=16, sr_seed=0)
+    return oracle.decode(state, fmt).reshape(N).astype(np.float64)
+
+
+@pytest.mark.parametrize("rule", [RTN, SR, WEYL])
+@pytest.mark.parametrize("sign", [+1, -1])
+def test_proposition_1_identity_end_to_end(rule, sign):
+    # a_t = 1, w_t = w, h_0 on the grid: h_T = h_0 + s*(T*m + #{t <= T : u_t >= 1 - f}), so
+    # e_T = -s*(#{u_t < 1 - f} - T(1 - f)).  All sums are exact in FP32 for these w (few bits).
+    step, T = 2.0**-10, 400
+    fracs = np.array([1, 3, 5, 8, 13, 16, 21, 27, 31, 33, 40, 47, 50, 55, 60, 63]) / 64.0
+    if sign > 0:
+        w, h0 = fracs, 1.0                                   # climbs inside [1, 2): spacing stays 2^-10
+    else:
+        w, h0 = -fracs, 1.0 + 1000 * step                    # descends inside [1, 2)
+    got = run_scalar_recurrence(w, h0, T, rule)
+    m = np.floor(w)
+    f = w - m
+    for n in range(16):
+        U = [oracle.threshold(rule, flat=n, t=t, weyl_block=16, sr_seed=0) for t in range(1, T + 1)]
+        if rule == RTN:
+            ups = T if f[n] > 0.5 else 0
+        else:
+            ups = sum(Fraction(u, 1 << 24) >= 1 - Fraction(float(f[n])) for u in U)
+        assert got[n] == h0 + step * (T * m[n] + ups)
+    err = (got - (h0 + step * T * w)) / step
+    if rule == RTN:       # Corollary 1(a): |e_T| = s T min(f, 1 - f)
+        assert np.allclose(np.abs(err), T * np.minimum(f, 1 - f))
+    elif rule == WEYL:    # Corollary 1(c): O(log T), far below RTN's linear growth
+        assert np.max(np.abs(err)) <= 4.0
+    else:                 # Corollary 1(b): typical size sqrt(T f (1 - f))
+        assert np.max(np.abs(err) / np.sqrt(T * f * (1 - f))) < 4.5
+
+
+def test_lemma_1_write_erasure_under_rtn():
+    # |delta| < s/2 on a grid value: RTN never moves the stored bits, SR and Weyl do.
+    step, T = 2.0**-10, 256
+    w = np.full(16, 0.3)
+    for rule, moved in ((RTN, False), (SR, True), (WEYL, True)):
+        got = run_scalar_recurrence(w, 1.0, T, rule)
+        assert np.all(got == 1.0) != moved
+        if moved:
+            assert np.all(np.abs(got - (1.0 + 0.3 * step * T)) < 0.3 * step * T * 0.5)
+
+
+# ---- Eq. 1 without rounding = textbook closed form --------------------------------------------
+def test_fp32_twin_matches_closed_form_in_double():
+    cfg = workloads.CONFIGS[1]
+    A, D = workloads.layer_params(cfg)
+    B_, H, P, N = cfg.state_shape
+    T = 48
+    state = np.zeros(cfg.state_shape, dtype=np.uint32)
+    ins = [workloads.step_inputs(cfg, t) for t in range(1, T + 1)]
+    for t, (x, dt, Bm, Cm) in enumerate(ins, start=1):
+        y = oracle.state_update(state, None, FP32, 0, x, dt, A, Bm, Cm, D, RTN, t)
+    # h_T = sum_t (prod_{k>t} a_k) w_t, y_T = C_T . h_T + D x_T, all in float64
+    a = [np.exp(dt.astype(np.float64) * A.astype(np.float64)[None, :]) for (_, dt, _, _) in ins]
+    h = np.zeros(cfg.state_shape)
+    for t, (x, dt, Bm, Cm) in enumerate(ins):
+        wt = (dt.astype(np.float64)[:, :, None] * x)[..., None] * Bm.astype(np.float64)[:, None, None, :]
+        decay = np.ones((B_, H))
+        for k in range(t + 1, T):
+            decay = decay * a[k]
+        h += decay[:, :, None, None] * wt
+    got = state.view(np.float32).astype(np.float64)
+    assert np.max(np.abs(got - h)) <= T * 2.0**-22 * np.max(np.abs(h))
+    x, dt, Bm, Cm = ins[-1]
+    y_ref = np.einsum("bhpn,bn->bhp", h, Cm.astype(np.float64)) + D.astype(np.float64)[None, :, None] * x
+    assert np.max(np.abs(y - y_ref)) <= 1e-5 * np.max(np.abs(y_ref))
+
+
+# ---- E4M3 block scale -------------------------------------------------------------------------
+def test_e4m3_scale_absorbs_a_shared_decay():
+    # With w = 0 and one decay per row the FP32 scale carries the decay and the codes stay put
+    # under RTN (a consequence of s = max|h| / 448 being recomputed at every write).
+    rng = np.random.default_rng(5)
+    shape = (1, 2, 4, 128)
+    src = rng.standard_normal(shape).astype(np.float32).reshape(-1, 128)
+    codes, scales = oracle.quantize_store(src, E4M3, RTN, 1, scale_block=128, weyl_block=128)
+    state = codes.reshape(shape).copy()
+    sc = scales.reshape(-1).copy()
+    assert np.allclose(sc, np.abs(src).max(axis=1) / 448.0, rtol=1e-6)
+    assert np.all(np.abs(oracle.decode(state, E4M3)).reshape(-1, 128).max(axis=1) == 448.0)
+    A = np.array([-0.5, -0.01], np.float32)
+    x = np.zeros((1, 2, 4), np.float32)
+    dt = np.full((1, 2), 0.1, np.float32)
+    z = np.zeros((1, 128), np.float32)
+    before, s_before = state.copy(), sc.copy()
+    for t in range(1, 20):
+        oracle.state_update(state, sc, E4M3, 128, x, dt, A, z, z, None, RTN, t, weyl_block=128)
+    assert np.array_equal(state, before)
+    a = np.exp(0.1 * A.astype(np.float64)) ** 19
+    ratio = (sc / s_before).reshape(2, 4)
+    assert np.allclose(ratio, a[:, None], rtol=1e-5)
+
+
+def test_zero_block_scale_is_the_smallest_normal():
+    codes, scales = oracle.quantize_store(np.zeros((1, 16), np.float32), E4M3, WEYL, 1, scale_block=16)
+    assert np.all(codes == 0) and scales[0, 0] == np.finfo(np.float32).tiny
+
+
+# ---- independent brute-force restatement on tiny states ----------------------------------------
+def grid_neighbours_round(v, U, fmt, rule, grid, max_finite):
+    """Eq. 2 on an enumerated grid (see test_oracle_rounding); RTN = nearest, ties to even code."""
+    if abs(v) > max_finite:
+        return float(np.copysign(max_finite, v))
+    i = int(np.searchsorted(grid, v, side="right")) - 1
+    lo = grid[i]
+    if lo == v:
+        return float(v)
+    hi = grid[i + 1]
+    f = (Fraction(float(v)) - Fraction(float(lo))) / (Fraction(float(hi)) - Fraction(float(lo)))
+    if rule == RTN:
+        if f != Fraction(1, 2):
+            return float(hi if f > Fraction(1, 2) else lo)
+        lo_code = int(oracle.encode(np.float32(lo), fmt)[0])
+        return float(lo if lo_code % 2 == 0 else hi)
+    return float(hi if Fraction(U, 1 << 24) >= 1 - f else lo)
+
+
+@pytest.mark.parametrize("fmt", [FP16, BF16, E4M3])
+@pytest.mark.parametrize("rule", [RTN, SR, WEYL])
+@pytest.mark.parametrize("a_per_state", [False, True])
+def test_update_against_python_restatement_on_tiny_state(fmt, rule, a_per_state):
+    from test_oracle_rounding import grid_of, MAX_FINITE
+    rng = np.random.default_rng(100 + 10 * fmt + rule)
+    Bsz, H, P, N = 2, 3, 2, 32
+    wb = 16
+    sb = 16 if fmt == E4M3 else 0
+    grid = grid_of(fmt)
+    f32 = np.float32
+    src = (rng.standard_normal((Bsz * H * P, N)) * 0.05).astype(f32)
+    codes, scales = oracle.quantize_store(src, fmt, RTN, 1, scale_block=sb, weyl_block=wb)
+    state = codes.reshape(Bsz, H, P, N).copy()
+    sc = None if scales is None else scales.reshape(-1).copy()
+    A = -np.exp(rng.uniform(-3, 1, (H, N) if a_per_state else (H,))).astype(f32)
+    D = rng.normal(0, 0.1, H).astype(f32)
+    base = 3
+    for t in (1, 2, 3):
+        x = rng.standard_normal((Bsz, H, P)).astype(f32)
+        dt = np.log1p(np.exp(rng.normal(-2, 0.5, (Bsz, H)))).astype(f32)
+        Bm = rng.standard_normal((Bsz, N)).astype(f32)
+        Cm = rng.standard_normal((Bsz, N)).astype(f32)
+        h_in = oracle.decode(state, fmt)
+        if fmt == E4M3:
+            h_in = (h_in.reshape(-1, sb) * sc[:, None]).astype(f32).reshape(state.shape)
+        want_codes = np.zeros_like(state)
+        want_scales = None if sc is None else np.zeros_like(sc)
+        want_y = np.zeros((Bsz, H, P))
+        for b in range(Bsz):
+            for h in range(H):
+                for p in range(P):
+                    dtx = f32(dt[b, h] * x[b, h, p])
+                    hp = np.zeros(N, f32)
+                    for n in range(N):
+                        Av = A[h, n] if a_per_state else A[h]
+                        a = oracle.exp_spec(f32(dt[b, h] * Av))[0]
+                        w = f32(dtx * Bm[b, n])
+                        # fused multiply-add: exact product and sum, one rounding
+                        hp[n] = f32(float(Fraction(float(a)) * Fraction(float(h_in[b, h, p, n])) + Fraction(float(w))))
+                    want_y[b, h, p] = float(np.dot(Cm[b].astype(np.float64), hp.astype(np.float64))
+                                            + float(D[h]) * float(x[b, h, p]))
+                    for k0 in range(0, N, 16):
+                        blk = hp[k0:k0 + 16]
+                        rinv = f32(1.0)
+                        if fmt == E4M3:
+                            s = max(f32(np.max(np.abs(blk)) / f32(448.0)), np.finfo(f32).tiny)
+                            rinv = f32(f32(1.0) / s)
+                            want_scales[(((b * H + h) * P + p) * N + k0) // 16] = s
+                        for j in range(16):
+                            n = k0 + j
+                            flat = ((((base + b) * H + h) * P + p) * N + n)
+                            if rule == WEYL:
+                                U = oracle.weyl_u24(flat // wb, flat % wb, 2, 1, t)
+                            elif rule == SR:
+                                g = flat // 4
+                                U = int(oracle.philox4x32_10([g, 0, t, 2], [9, 0])[flat % 4]) >> 8
+                            else:
+                                U = 0
+                            v = f32(blk[j] * rinv) if fmt == E4M3 else blk[j]
+                            q = grid_neighbours_round(float(v), U, fmt, rule, grid, MAX_FINITE[fmt])
+                            want_codes[b, h, p, n] = oracle.encode(f32(q), fmt)[0]
+                            if q == 0.0 and np.signbit(v):
+                                want_codes[b, h, p, n] = oracle.encode(f32(-0.0), fmt)[0]
+        y = oracle.state_update(state, sc, fmt, sb, x, dt, A, Bm, Cm, D, rule, t, layer=2, weyl_seed=1,
+                                weyl_block=wb, sr_seed=9, batch_index_base=base)
+        assert np.array_equal(state, want_codes)
+        if sc is not None:
+            assert np.array_equal(sc, want_scales)
+        assert np.allclose(y, want_y, rtol=0, atol=1e-6 * np.max(np.abs(want_y)))
+
+
+def test_sharding_invariance_of_indices():
+    # a batch slice updated with batch_index_base reproduces the same rows of the full batch
+    cfg = workloads.CONFIGS[1].with_batch(4)
+    A, D = workloads.layer_params(cfg)
+    for rule in (SR, WEYL):
+        full, _ = oracle.new_state(cfg.state_shape, FP16)
+        part = full[2:].copy()
+        for t in range(1, 6):
+            x, dt, Bm, Cm = workloads.step_inputs(cfg, t)
+            y = oracle.state_update(full, None, FP16, 0, x, dt, A, Bm, Cm, D, rule, t)
+            y2 = oracle.state_update(part, None, FP16, 0, x[2:], dt[2:], A, Bm[2:], Cm[2:], D, rule, t,
+                                     batch_index_base=2)
+            assert np.array_equal(full[2:], part) and np.array_equal(y[2:], y2)
