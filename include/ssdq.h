@@ -1,0 +1,151 @@
+/* ssdq.h -- C ABI of the quantized selective-state-update decode library (CUDA, sm_100a).
+ *
+ * The library keeps a Mamba-style recurrent state in a low-precision store (FP16, BF16 or
+ * FP8-E4M3 with an FP32 block scale) and, once per generated token and layer, makes one fused
+ * pass over it: dequantise, h' = exp(dt*A)*h + dt*B*x (Eq. 1; Appendix B "Runners"), read out
+ * y = C.h' + D*x from the unrounded h', and write h' back rounded by Eq. 2 under one of three
+ * threshold rules (Section 2 "Rounding with a threshold"): round-to-nearest, stochastic rounding
+ * driven by counter-based Philox4x32-10, or the golden-ratio Weyl dither in its 32-bit integer form
+ * (Appendix B "Dithers").
+ *
+ * Conventions for every entry point
+ *   - Pointers named in a descriptor are DEVICE pointers unless stated; descriptors themselves are
+ *     HOST memory and are copied by value at launch.  The caller owns all memory.  Unless an entry
+ *     point says otherwise the library allocates nothing on the device.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls enqueue
+ *     work and return; they do not synchronise.
+ *   - Every argument check happens before any launch; a failed check launches nothing.
+ *   - Return value: SSDQ_OK or a negative ssdq_status; ssdq_last_error() gives a thread-local text.
+ *   - Indices that feed the thresholds are GLOBAL: entry (b, h, p, n) of a layer has flat index
+ *     ((( b + batch_index_base) * H + h) * P + p) * N + n, so a batch shard reproduces the bits of
+ *     the unsharded run.
+ *   - All inputs must be finite.  Binary32 subnormals are honoured (no flush to zero).
+ */
+#ifndef SSDQ_H_
+#define SSDQ_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SSDQ_OK = 0,
+    SSDQ_ERR_NULL = -1,         /* a required pointer is NULL */
+    SSDQ_ERR_SHAPE = -2,        /* a size is zero or inconsistent */
+    SSDQ_ERR_ALIGN = -3,        /* a pointer is not aligned as documented */
+    SSDQ_ERR_UNSUPPORTED = -4,  /* a valid request this build has no kernel for */
+    SSDQ_ERR_CUDA = -5          /* the CUDA runtime reported an error (see ssdq_last_error) */
+} ssdq_status;
+
+/* Storage formats (Appendix B "Formats").  SSDQ_FP32 stores binary32 and never rounds: it is the
+ * full-precision twin that the quantised trajectory is compared with. */
+typedef enum { SSDQ_FP16 = 0, SSDQ_BF16 = 1, SSDQ_E4M3 = 2, SSDQ_FP32 = 3 } ssdq_format;
+
+/* Threshold rules of Eq. 2.  RTN rounds to nearest, ties to even (the rule of native casts). */
+typedef enum { SSDQ_RTN = 0, SSDQ_SR_PHILOX = 1, SSDQ_WEYL = 2 } ssdq_rule;
+
+/* Weyl dither in 32-bit fixed point (Appendix B "Dithers", hardware form):
+ *   acc(r, c, t) = mul_row*(r+1) + mul_col*(c+1) + base + t*phi   (mod 2^32),   u = (acc >> 8) / 2^24
+ * with r = flat / block and c = flat % block.  Plain data, 32 bytes, no pointers. */
+typedef struct {
+    uint32_t mul_row;   /* 0.7548776662 * 2^32 */
+    uint32_t mul_col;   /* 0.5698402910 * 2^32 */
+    uint32_t phi;       /* 2654435769, the golden-ratio increment */
+    uint32_t base;      /* 0.1234567*2^32 * layer + 0.3141592*2^32 * seed  (mod 2^32) */
+    uint32_t block;     /* entries per dither block along the state dimension: 16, or N */
+    uint32_t layer;
+    uint32_t seed;
+    uint32_t reserved;
+} ssdq_weyl;
+
+/* Fill `out` (HOST) for layer `layer` and offset seed `seed` (the paper's sigma; 0 in its runs).
+ * `block` must be a positive multiple of 16.  Pure host arithmetic; no CUDA call. */
+int weyl_offsets_init(ssdq_weyl* out, uint32_t layer, uint32_t seed, uint32_t block);
+
+/* Test aid: write the 24-bit thresholds U of entries flat = first_flat .. first_flat + n - 1 at
+ * write index step_t into out_u24 (DEVICE, n x uint32).  rule = SSDQ_WEYL uses `weyl`;
+ * SSDQ_SR_PHILOX uses Philox4x32-10 with key = sr_seed and counter = (flat/4 low, flat/4 high,
+ * step_t, layer), word flat % 4, top 24 bits; SSDQ_RTN writes zeros. */
+int ssdq_thresholds_materialize(int rule, const ssdq_weyl* weyl, uint64_t sr_seed, uint32_t layer,
+                                uint64_t first_flat, uint64_t n, uint32_t step_t, uint32_t* out_u24, void* stream);
+
+/* One layer's decode-step problem. */
+typedef struct {
+    uint32_t batch, nheads, headdim, dstate;  /* B, H, P, N.  N in {16, 32, 64, 128, 256} (E4M3: N >= 16;
+                                                 FP32: N >= 16).  Mamba-1 is H = d_inner, P = 1. */
+    void* state;         /* [B, H, P, N] codes of `format`, N contiguous, 16-byte aligned; updated IN PLACE */
+    float* scales;       /* E4M3 only: [B, H, P, N / scale_block] FP32 block scales, updated in place */
+    uint32_t scale_block;/* E4M3 only: 16 or N (entries along N that share one scale) */
+    int32_t format;      /* ssdq_format */
+    const float* x;      /* [B, H, P] */
+    const float* dt;     /* [B, H], already passed through softplus */
+    const float* A;      /* [H] (one decay per head) or [H, N] if a_per_state; [H, N] must be 16-byte aligned */
+    const float* Bm;     /* [B, N], one group, 16-byte aligned */
+    const float* Cm;     /* [B, N], one group, 16-byte aligned */
+    const float* D;      /* [H] or NULL (no skip term) */
+    uint32_t a_per_state;/* 0: A is [H]; 1: A is [H, N] (Mamba-1) */
+    float* y;            /* [B, H, P] output */
+    int32_t rule;        /* ssdq_rule */
+    ssdq_weyl weyl;      /* used when rule == SSDQ_WEYL; weyl.block must be 16 or N */
+    uint64_t sr_seed;    /* Philox key when rule == SSDQ_SR_PHILOX */
+    uint32_t layer;      /* layer index in the SR counter (the Weyl layer term sits in weyl.base) */
+    uint32_t batch_index_base;  /* global index of local sequence 0 */
+} ssdq_update_desc;
+
+/* One fused decode step of one layer (Eq. 1, readout, Eq. 2), in place, one kernel launch:
+ *   h  = dequant(state)                          (E4M3: code * scale, one rounded multiply)
+ *   a  = exp_spec(dt*A);  w = (dt*x)*B;  h' = fma(a, h, w)      all binary32, in this order
+ *   y  = sum_n C[n]*h'[n] + D*x                  (FP32 accumulation, tree order unspecified)
+ *   E4M3: s = max(amax_block(h') / 448, FLT_MIN), v = h' * (1/s);  otherwise v = h'
+ *   state = encode(Q_u(v)) with u from `rule` at write index step_t (first write is step_t = 1)
+ * exp_spec is the library's fixed binary32 exponential (clamp to [-87, 88], Cody-Waite reduction,
+ * degree-7 polynomial), identical bit for bit on every call.  Values beyond the format's largest
+ * finite number saturate to it; a value rounded to zero keeps its sign. */
+int ssd_state_update(const ssdq_update_desc* d, uint32_t step_t, void* stream);
+
+/* Quantise an FP32 array into a store with the same rounding functions (Eq. 2): used to seed h_0
+ * from a full-precision state (the paper quantises the end-of-prefill state) and to exercise the
+ * rules in isolation.  src [n_rows, row_len] DEVICE floats (16-byte aligned); dst_codes
+ * [n_rows, row_len] codes (16-byte aligned); dst_scales [n_rows, row_len / scale_block] for E4M3
+ * else NULL.  row_len obeys the same limits as dstate; entry (row, col) has flat index
+ * (row_index_base + row) * row_len + col. */
+int quantize_store(const float* src, void* dst_codes, float* dst_scales, uint64_t n_rows, uint32_t row_len,
+                   uint32_t scale_block, int format, int rule, const ssdq_weyl* weyl, uint64_t sr_seed,
+                   uint32_t layer, uint64_t row_index_base, uint32_t step_t, void* stream);
+
+/* Inverse view of a store: out[i] = decode(code[i]) (* scale[i / scale_block] for E4M3), DEVICE. */
+int ssdq_dequantize(const void* codes, const float* scales, uint64_t n, int format, uint32_t scale_block,
+                    float* out, void* stream);
+
+/* Per-step inputs of the multi-step driver: element (t, l) of tensor X starts at
+ * X + (((t - t_first) % ring) * n_layers + l) * stride_X floats, all DEVICE memory. */
+typedef struct {
+    const float* x;   uint64_t stride_x;    /* each [B, H, P] */
+    const float* dt;  uint64_t stride_dt;   /* each [B, H] */
+    const float* Bm;  uint64_t stride_B;    /* each [B, N] */
+    const float* Cm;  uint64_t stride_C;    /* each [B, N] */
+    float* y;         uint64_t stride_y;    /* each [B, H, P]; written for every (t, l) slot of the ring */
+    uint32_t ring;    /* number of distinct steps stored (>= 1; == n_steps when every step has its own inputs) */
+    uint32_t reserved;
+} ssdq_step_inputs;
+
+/* T-step decode driver (the open-loop replay of Appendix B run forward): for t = t_first ..
+ * t_first + n_steps - 1 and l = 0 .. n_layers - 1, one ssd_state_update launch of layers[l] with
+ * write index t and the inputs of slot (t, l), all on `stream`, no host synchronisation.  The
+ * x / dt / Bm / Cm / y members of layers[l] are ignored (taken from `in`). */
+int ssd_decode_run(const ssdq_update_desc* layers, uint32_t n_layers, uint32_t t_first, uint32_t n_steps,
+                   const ssdq_step_inputs* in, void* stream);
+
+/* Text of the last error on this thread ("" if none).  The pointer stays valid until the next call
+ * of the library on the same thread. */
+const char* ssdq_last_error(void);
+
+/* Number of kernels the library has launched in this process (a counter for benchmarks). */
+uint64_t ssdq_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SSDQ_H_ */

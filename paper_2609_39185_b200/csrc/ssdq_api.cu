@@ -1,0 +1,222 @@
+// ssdq_api.cu -- the C ABI declared in include/ssdq.h: argument checks, then one launch per call
+// (one per layer and step for the multi-step driver).  No device allocation, no global state
+// besides a thread-local error text and a launch counter.
+#include <atomic>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+
+#include "../../include/ssdq.h"
+#include "ssdq_internal.h"
+
+namespace {
+
+thread_local char g_err[256] = "";
+std::atomic<uint64_t> g_launches{0};
+
+int fail(int code, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+int cuda_result(cudaError_t e, const char* what) {
+    if (e == cudaSuccess) { g_launches.fetch_add(1, std::memory_order_relaxed); return SSDQ_OK; }
+    return fail(SSDQ_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
+
+bool dstate_supported(int fmt, uint32_t n) {
+    if (!(n == 16 || n == 32 || n == 64 || n == 128 || n == 256)) return false;
+    if (fmt == SSDQ_FP32 && n > 128) return false;   // a row of 256 floats would span two warps
+    return true;
+}
+
+ssdq::WeylConst weyl_const(const ssdq_weyl& w) {
+    return ssdq::WeylConst{w.mul_row, w.mul_col, w.phi, w.base, w.block};
+}
+
+// Checks shared by ssd_state_update and ssd_decode_run; per-step pointers are checked separately.
+int check_layer(const ssdq_update_desc* d) {
+    if (!d) return fail(SSDQ_ERR_NULL, "descriptor is NULL");
+    if (d->batch == 0 || d->nheads == 0 || d->headdim == 0) return fail(SSDQ_ERR_SHAPE, "batch, nheads and headdim must be positive");
+    if (d->format < SSDQ_FP16 || d->format > SSDQ_FP32) return fail(SSDQ_ERR_UNSUPPORTED, "unknown format %d", d->format);
+    if (d->rule < SSDQ_RTN || d->rule > SSDQ_WEYL) return fail(SSDQ_ERR_UNSUPPORTED, "unknown rule %d", d->rule);
+    if (!dstate_supported(d->format, d->dstate)) return fail(SSDQ_ERR_UNSUPPORTED, "dstate %u is not supported for format %d", d->dstate, d->format);
+    if ((uint64_t)d->batch * d->nheads > 0xFFFFFFFFull / 2) return fail(SSDQ_ERR_SHAPE, "batch * nheads too large");
+    if (!d->state || !d->A) return fail(SSDQ_ERR_NULL, "state and A are required");
+    if (!aligned16(d->state)) return fail(SSDQ_ERR_ALIGN, "state must be 16-byte aligned");
+    if (d->a_per_state ? !aligned16(d->A) : !aligned4(d->A)) return fail(SSDQ_ERR_ALIGN, "A is misaligned");
+    if (d->D && !aligned4(d->D)) return fail(SSDQ_ERR_ALIGN, "D is misaligned");
+    if (d->format == SSDQ_E4M3) {
+        if (!d->scales) return fail(SSDQ_ERR_NULL, "E4M3 needs a scale array");
+        if (!aligned4(d->scales)) return fail(SSDQ_ERR_ALIGN, "scales are misaligned");
+        if (d->scale_block == (uint32_t)d->headdim * d->dstate && d->scale_block != d->dstate)
+            return fail(SSDQ_ERR_UNSUPPORTED, "one scale per head is not built; use scale_block 16 or dstate");
+        if (!(d->scale_block == 16 || d->scale_block == d->dstate)) return fail(SSDQ_ERR_SHAPE, "scale_block must be 16 or dstate");
+    }
+    if (d->rule == SSDQ_WEYL && d->format != SSDQ_FP32) {
+        if (!(d->weyl.block == 16 || d->weyl.block == d->dstate)) return fail(SSDQ_ERR_SHAPE, "weyl.block must be 16 or dstate");
+        if (d->weyl.phi == 0 || (d->weyl.phi & 1u) == 0) return fail(SSDQ_ERR_SHAPE, "weyl descriptor is not initialised");
+    }
+    return SSDQ_OK;
+}
+
+int check_step_ptrs(const float* x, const float* dt, const float* Bm, const float* Cm, const float* y) {
+    if (!x || !dt || !Bm || !Cm || !y) return fail(SSDQ_ERR_NULL, "x, dt, Bm, Cm and y are required");
+    if (!aligned4(x) || !aligned4(dt) || !aligned4(y)) return fail(SSDQ_ERR_ALIGN, "x, dt or y is misaligned");
+    if (!aligned16(Bm) || !aligned16(Cm)) return fail(SSDQ_ERR_ALIGN, "Bm and Cm must be 16-byte aligned");
+    return SSDQ_OK;
+}
+
+ssdq::UpdateParams make_params(const ssdq_update_desc* d, uint32_t step_t) {
+    ssdq::UpdateParams p{};
+    p.state = d->state; p.scales = d->scales;
+    p.x = d->x; p.dt = d->dt; p.A = d->A; p.Bm = d->Bm; p.Cm = d->Cm; p.D = d->D; p.y = d->y;
+    p.B = d->batch; p.H = d->nheads; p.P = d->headdim; p.N = d->dstate;
+    p.n_items = d->batch * d->nheads;
+    p.scale_block = d->scale_block;
+    p.step_t = step_t; p.layer = d->layer; p.batch_base = d->batch_index_base;
+    p.weyl = weyl_const(d->weyl);
+    p.sr_seed = d->sr_seed;
+    return p;
+}
+
+cudaError_t launch_update(const ssdq::UpdateParams& p, int fmt, int rule, bool aps, cudaStream_t s) {
+    switch (fmt) {
+        case SSDQ_FP16: return ssdq::launch_update_fp16(p, rule, aps, s);
+        case SSDQ_BF16: return ssdq::launch_update_bf16(p, rule, aps, s);
+        case SSDQ_E4M3: return ssdq::launch_update_e4m3(p, rule, aps, s);
+        case SSDQ_FP32: return ssdq::launch_update_fp32(p, rule, aps, s);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace
+
+extern "C" {
+
+int weyl_offsets_init(ssdq_weyl* out, uint32_t layer, uint32_t seed, uint32_t block) {
+    if (!out) return fail(SSDQ_ERR_NULL, "out is NULL");
+    if (block == 0 || block % 16 != 0) return fail(SSDQ_ERR_SHAPE, "block must be a positive multiple of 16");
+    // Appendix B "Dithers": the decimal generators times 2^32, rounded to the nearest integer.
+    const uint32_t kRow = 3242174889u, kCol = 2447445414u, kLayer = 530242489u, kSeed = 1349303490u;
+    out->mul_row = kRow;
+    out->mul_col = kCol;
+    out->phi = 2654435769u;
+    out->base = kLayer * layer + kSeed * seed;
+    out->block = block;
+    out->layer = layer;
+    out->seed = seed;
+    out->reserved = 0;
+    g_err[0] = 0;
+    return SSDQ_OK;
+}
+
+int ssdq_thresholds_materialize(int rule, const ssdq_weyl* weyl, uint64_t sr_seed, uint32_t layer, uint64_t first_flat,
+                                uint64_t n, uint32_t step_t, uint32_t* out_u24, void* stream) {
+    if (rule < SSDQ_RTN || rule > SSDQ_WEYL) return fail(SSDQ_ERR_UNSUPPORTED, "unknown rule %d", rule);
+    if (n && !out_u24) return fail(SSDQ_ERR_NULL, "out_u24 is NULL");
+    ssdq::WeylConst w{};
+    if (rule == SSDQ_WEYL) {
+        if (!weyl) return fail(SSDQ_ERR_NULL, "weyl descriptor is NULL");
+        if (weyl->block == 0) return fail(SSDQ_ERR_SHAPE, "weyl.block is zero");
+        w = weyl_const(*weyl);
+    }
+    if (n == 0) return SSDQ_OK;
+    return cuda_result(ssdq::launch_thresholds(rule, w, sr_seed, layer, first_flat, n, step_t, out_u24,
+                                               static_cast<cudaStream_t>(stream)), "thresholds kernel");
+}
+
+int ssd_state_update(const ssdq_update_desc* d, uint32_t step_t, void* stream) {
+    int rc = check_layer(d);
+    if (rc != SSDQ_OK) return rc;
+    rc = check_step_ptrs(d->x, d->dt, d->Bm, d->Cm, d->y);
+    if (rc != SSDQ_OK) return rc;
+    const ssdq::UpdateParams p = make_params(d, step_t);
+    return cuda_result(launch_update(p, d->format, d->rule, d->a_per_state != 0, static_cast<cudaStream_t>(stream)),
+                       "state-update kernel");
+}
+
+int quantize_store(const float* src, void* dst_codes, float* dst_scales, uint64_t n_rows, uint32_t row_len,
+                   uint32_t scale_block, int format, int rule, const ssdq_weyl* weyl, uint64_t sr_seed, uint32_t layer,
+                   uint64_t row_index_base, uint32_t step_t, void* stream) {
+    if (format < SSDQ_FP16 || format > SSDQ_FP32) return fail(SSDQ_ERR_UNSUPPORTED, "unknown format %d", format);
+    if (rule < SSDQ_RTN || rule > SSDQ_WEYL) return fail(SSDQ_ERR_UNSUPPORTED, "unknown rule %d", rule);
+    if (!dstate_supported(format, row_len)) return fail(SSDQ_ERR_UNSUPPORTED, "row_len %u is not supported for format %d", row_len, format);
+    if (n_rows == 0) return SSDQ_OK;
+    if (!src || !dst_codes) return fail(SSDQ_ERR_NULL, "src and dst_codes are required");
+    if (!aligned16(src) || !aligned16(dst_codes)) return fail(SSDQ_ERR_ALIGN, "src and dst_codes must be 16-byte aligned");
+    ssdq::QuantParams p{};
+    if (format == SSDQ_E4M3) {
+        if (!dst_scales) return fail(SSDQ_ERR_NULL, "E4M3 needs a scale array");
+        if (!(scale_block == 16 || scale_block == row_len)) return fail(SSDQ_ERR_SHAPE, "scale_block must be 16 or row_len");
+    }
+    if (rule == SSDQ_WEYL && format != SSDQ_FP32) {
+        if (!weyl) return fail(SSDQ_ERR_NULL, "weyl descriptor is NULL");
+        if (!(weyl->block == 16 || weyl->block == row_len)) return fail(SSDQ_ERR_SHAPE, "weyl.block must be 16 or row_len");
+        p.weyl = weyl_const(*weyl);
+    }
+    p.src = src; p.codes = dst_codes; p.scales = dst_scales; p.n_rows = n_rows; p.row_len = row_len;
+    p.scale_block = scale_block; p.step_t = step_t; p.layer = layer; p.row_base = row_index_base; p.sr_seed = sr_seed;
+    return cuda_result(ssdq::launch_quantize(p, format, rule, static_cast<cudaStream_t>(stream)), "quantize kernel");
+}
+
+int ssdq_dequantize(const void* codes, const float* scales, uint64_t n, int format, uint32_t scale_block, float* out,
+                    void* stream) {
+    if (format < SSDQ_FP16 || format > SSDQ_FP32) return fail(SSDQ_ERR_UNSUPPORTED, "unknown format %d", format);
+    if (n == 0) return SSDQ_OK;
+    if (!codes || !out) return fail(SSDQ_ERR_NULL, "codes and out are required");
+    if (n % 16 != 0) return fail(SSDQ_ERR_SHAPE, "n must be a multiple of 16");
+    if (!aligned16(codes) || !aligned16(out)) return fail(SSDQ_ERR_ALIGN, "codes and out must be 16-byte aligned");
+    if (format == SSDQ_E4M3 && (!scales || scale_block == 0 || scale_block % 16 != 0))
+        return fail(SSDQ_ERR_SHAPE, "E4M3 needs scales and a scale_block that is a multiple of 16");
+    return cuda_result(ssdq::launch_dequantize(codes, scales, n, format, scale_block, out, static_cast<cudaStream_t>(stream)),
+                       "dequantize kernel");
+}
+
+int ssd_decode_run(const ssdq_update_desc* layers, uint32_t n_layers, uint32_t t_first, uint32_t n_steps,
+                   const ssdq_step_inputs* in, void* stream) {
+    if (!layers || !in) return fail(SSDQ_ERR_NULL, "layers and in are required");
+    if (n_layers == 0 || in->ring == 0) return fail(SSDQ_ERR_SHAPE, "n_layers and ring must be positive");
+    for (uint32_t l = 0; l < n_layers; ++l) {
+        const int rc = check_layer(&layers[l]);
+        if (rc != SSDQ_OK) return rc;
+    }
+    // every slot of the ring is used with every layer: check the alignment of each (slot, layer) once
+    const uint32_t slots = n_steps < in->ring ? n_steps : in->ring;
+    for (uint32_t s = 0; s < slots; ++s)
+        for (uint32_t l = 0; l < n_layers; ++l) {
+            const uint64_t k = (uint64_t)s * n_layers + l;
+            const int rc = check_step_ptrs(in->x + k * in->stride_x, in->dt + k * in->stride_dt, in->Bm + k * in->stride_B,
+                                           in->Cm + k * in->stride_C, in->y + k * in->stride_y);
+            if (rc != SSDQ_OK) return rc;
+        }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    for (uint32_t i = 0; i < n_steps; ++i) {
+        const uint32_t t = t_first + i;
+        for (uint32_t l = 0; l < n_layers; ++l) {
+            const uint64_t k = (uint64_t)(i % in->ring) * n_layers + l;
+            ssdq::UpdateParams p = make_params(&layers[l], t);
+            p.x = in->x + k * in->stride_x;
+            p.dt = in->dt + k * in->stride_dt;
+            p.Bm = in->Bm + k * in->stride_B;
+            p.Cm = in->Cm + k * in->stride_C;
+            p.y = in->y + k * in->stride_y;
+            const int rc = cuda_result(launch_update(p, layers[l].format, layers[l].rule, layers[l].a_per_state != 0, s),
+                                       "state-update kernel");
+            if (rc != SSDQ_OK) return rc;
+        }
+    }
+    return SSDQ_OK;
+}
+
+const char* ssdq_last_error(void) { return g_err; }
+
+uint64_t ssdq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

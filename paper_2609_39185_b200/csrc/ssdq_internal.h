@@ -1,0 +1,60 @@
+// ssdq_internal.h -- host/device plain-data structures passed between the C ABI and the kernels.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include "ssdq_device.cuh"
+
+namespace ssdq {
+
+// Kernel parameters of one fused update launch (copied by value into constant memory at launch).
+struct UpdateParams {
+    void* state;
+    float* scales;
+    const float* x;
+    const float* dt;
+    const float* A;
+    const float* Bm;
+    const float* Cm;
+    const float* D;
+    float* y;
+    uint32_t B, H, P, N;
+    uint32_t n_items;        // B * H
+    uint32_t scale_block;    // E4M3: 16 or N
+    uint32_t step_t;
+    uint32_t layer;
+    uint32_t batch_base;
+    uint32_t spi;            // slots per (b, h) item inside a CTA (power of two)
+    uint32_t items_per_cta;
+    uint32_t rps;            // rows per slot
+    WeylConst weyl;
+    uint64_t sr_seed;
+};
+
+// Parameters of quantize_store / dequantize / thresholds.
+struct QuantParams {
+    const float* src;
+    void* codes;
+    float* scales;
+    uint64_t n_rows;
+    uint32_t row_len;
+    uint32_t scale_block;
+    uint32_t step_t;
+    uint32_t layer;
+    uint64_t row_base;
+    WeylConst weyl;
+    uint64_t sr_seed;
+};
+
+// one translation unit per storage format
+cudaError_t launch_update_fp16(const UpdateParams& p, int rule, bool a_per_state, cudaStream_t s);
+cudaError_t launch_update_bf16(const UpdateParams& p, int rule, bool a_per_state, cudaStream_t s);
+cudaError_t launch_update_e4m3(const UpdateParams& p, int rule, bool a_per_state, cudaStream_t s);
+cudaError_t launch_update_fp32(const UpdateParams& p, int rule, bool a_per_state, cudaStream_t s);
+
+cudaError_t launch_quantize(const QuantParams& p, int fmt, int rule, cudaStream_t s);
+cudaError_t launch_dequantize(const void* codes, const float* scales, uint64_t n, int fmt, uint32_t scale_block,
+                              float* out, cudaStream_t s);
+cudaError_t launch_thresholds(int rule, const WeylConst& w, uint64_t sr_seed, uint32_t layer, uint64_t first_flat,
+                              uint64_t n, uint32_t step_t, uint32_t* out, cudaStream_t s);
+
+}  // namespace ssdq

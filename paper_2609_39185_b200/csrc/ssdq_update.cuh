@@ -1,0 +1,305 @@
+// ssdq_update.cuh -- the fused decode-step kernel: dequantise -> Eq. 1 -> readout -> threshold ->
+// Eq. 2 -> encode -> store, one pass over the state, bounded by HBM bandwidth.
+//
+// Data layout and thread mapping.  The state is [B, H, P, N] with N contiguous; a row (b, h, p) is
+// N codes.  Each lane owns 16 bytes of a row (EPL = 8 two-byte codes, 16 E4M3 codes or 4 floats), so a
+// row is held by LPR = N / EPL neighbouring lanes (a "slot").  A CTA of kThreads lanes has
+// kThreads / LPR slots; they are split over `items_per_cta` (b, h) items, `spi` slots per item, and a
+// slot walks `rps` consecutive rows p of its item.  A lane therefore keeps its B[n], C[n] (and its
+// decays when A is per state) in registers for the whole CTA, issues UNR independent 128-bit loads
+// before it touches the first of them, and produces one partial dot per row which the slot reduces
+// with xor-shuffles.  Nothing is shared between CTAs, every state byte has one reader-then-writer.
+#pragma once
+#include "ssdq_device.cuh"
+#include "ssdq_internal.h"
+
+namespace ssdq {
+
+constexpr int kThreads = 128;
+
+template <int FMT> struct Unroll { static constexpr int value = 4; };
+template <> struct Unroll<FMT_E4M3> { static constexpr int value = 2; };
+
+// Unpack the lane's 16 bytes into EPL floats (exact widening; E4M3 is multiplied by its scale later).
+template <int FMT>
+__device__ __forceinline__ void unpack_lane(const uint4& raw, float* h) {
+    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+    if constexpr (FMT == FMT_FP16) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) unpack2_fp16(w[i], h[2 * i], h[2 * i + 1]);
+    } else if constexpr (FMT == FMT_BF16) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) unpack2_bf16(w[i], h[2 * i], h[2 * i + 1]);
+    } else if constexpr (FMT == FMT_E4M3) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) unpack4_e4m3(w[i], h + 4 * i);
+    } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) h[i] = __uint_as_float(w[i]);
+    }
+}
+
+// Round the lane's EPL values v[] under RULE and pack them into 16 bytes.
+// acc0: Weyl accumulator of the lane's first entry (RULE_WEYL); ctr/key: Philox counter of the
+// lane's first group of four entries (RULE_SR).
+template <int FMT, int RULE>
+__device__ __forceinline__ uint4 round_pack_lane(const float* v, uint32_t acc0, uint32_t mul_col, uint32_t g_lo,
+                                                 uint32_t g_hi, uint32_t step_t, uint32_t layer, uint32_t key0,
+                                                 uint32_t key1) {
+    constexpr int EPL = Fmt<FMT>::kEpl;
+    uint32_t w[4];
+    if constexpr (FMT == FMT_FP32) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) w[i] = __float_as_uint(v[i]);
+    } else if constexpr (RULE == RULE_RTN) {
+        if constexpr (FMT == FMT_FP16) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) w[i] = rtn_pack2_fp16(v[2 * i], v[2 * i + 1]);
+        } else if constexpr (FMT == FMT_BF16) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) w[i] = rtn_pack2_bf16(v[2 * i], v[2 * i + 1]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                w[i] = rtn_pack2_e4m3(v[4 * i], v[4 * i + 1]) | (rtn_pack2_e4m3(v[4 * i + 2], v[4 * i + 3]) << 16);
+        }
+    } else {
+        uint32_t acc[EPL];
+        if constexpr (RULE == RULE_WEYL) {
+#pragma unroll
+            for (int k = 0; k < EPL; ++k) acc[k] = acc0 + (uint32_t)k * mul_col;
+        } else {
+#pragma unroll
+            for (int g = 0; g < EPL / 4; ++g) {
+                const uint32_t lo = g_lo + (uint32_t)g;           // g_lo is a multiple of EPL / 4: no carry
+                const uint4 o = philox4x32_10(make_uint4(lo, g_hi, step_t, layer), key0, key1);
+                acc[4 * g] = o.x; acc[4 * g + 1] = o.y; acc[4 * g + 2] = o.z; acc[4 * g + 3] = o.w;
+            }
+        }
+        if constexpr (FMT == FMT_FP16) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                w[i] = dither_code_fp16(v[2 * i], acc[2 * i]) | (dither_code_fp16(v[2 * i + 1], acc[2 * i + 1]) << 16);
+        } else if constexpr (FMT == FMT_BF16) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                w[i] = dither_code_bf16(v[2 * i], acc[2 * i]) | (dither_code_bf16(v[2 * i + 1], acc[2 * i + 1]) << 16);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                w[i] = dither_code_e4m3(v[4 * i], acc[4 * i]) | (dither_code_e4m3(v[4 * i + 1], acc[4 * i + 1]) << 8) |
+                       (dither_code_e4m3(v[4 * i + 2], acc[4 * i + 2]) << 16) |
+                       (dither_code_e4m3(v[4 * i + 3], acc[4 * i + 3]) << 24);
+        }
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// Per-lane threshold set-up for the row with global index `grow` (row of the [B_global*H*P, N] view).
+template <int FMT, int RULE, int LPR>
+struct LaneThreshold {
+    static constexpr int EPL = Fmt<FMT>::kEpl;
+    static constexpr int N = LPR * EPL;
+    uint32_t lane_const;   // Weyl: everything but the row term
+    uint32_t row_mul;      // Weyl: mul_row * (dither blocks per row)
+    uint32_t n0;
+
+    __device__ __forceinline__ void init(const WeylConst& wc, uint32_t step_t, uint32_t lane_in_slot) {
+        n0 = lane_in_slot * EPL;
+        if constexpr (RULE == RULE_WEYL) {
+            // block == N: r = grow, c = n;   block == 16: r = grow * (N/16) + n / 16, c = n % 16
+            const bool row_block = (wc.block == (uint32_t)N);
+            const uint32_t blocks_per_row = row_block ? 1u : (uint32_t)N / 16u;
+            const uint32_t r_in_row = row_block ? 0u : n0 / 16u;
+            const uint32_t c0 = row_block ? n0 : n0 % 16u;
+            row_mul = wc.mul_row * blocks_per_row;
+            lane_const = wc.mul_row * (r_in_row + 1u) + wc.mul_col * (c0 + 1u) + wc.base + step_t * wc.phi;
+        }
+    }
+    __device__ __forceinline__ uint32_t weyl_acc0(uint64_t grow) const { return lane_const + row_mul * (uint32_t)grow; }
+    __device__ __forceinline__ void sr_group(uint64_t grow, uint32_t& g_lo, uint32_t& g_hi) const {
+        const uint64_t g = (grow * (uint64_t)N + n0) >> 2;
+        g_lo = (uint32_t)g;
+        g_hi = (uint32_t)(g >> 32);
+    }
+};
+
+template <int FMT, int RULE, int LPR, bool APS>
+__global__ void __launch_bounds__(kThreads) ssd_update_kernel(const UpdateParams p) {
+    constexpr int EPL = Fmt<FMT>::kEpl;
+    constexpr int N = LPR * EPL;
+    constexpr int UNR = Unroll<FMT>::value;
+    constexpr unsigned FULL = 0xFFFFFFFFu;
+
+    const uint32_t tid = threadIdx.x;
+    const uint32_t lis = tid % LPR;                 // lane in slot
+    const uint32_t slot = tid / LPR;
+    const uint32_t item_raw = blockIdx.x * p.items_per_cta + slot / p.spi;
+    const uint32_t sub = slot % p.spi;
+    const bool item_ok = item_raw < p.n_items;
+    const uint32_t item = item_ok ? item_raw : p.n_items - 1u;   // clamp: idle lanes still shuffle
+    const uint32_t b = item / p.H;
+    const uint32_t h = item - b * p.H;
+    const uint32_t n0 = lis * EPL;
+
+    // lane constants: B[n], C[n], decay(s), dt, D
+    float Bv[EPL], Cv[EPL];
+    {
+        const float4* Bp = reinterpret_cast<const float4*>(p.Bm + (size_t)b * N + n0);
+        const float4* Cp = reinterpret_cast<const float4*>(p.Cm + (size_t)b * N + n0);
+#pragma unroll
+        for (int i = 0; i < EPL / 4; ++i) {
+            const float4 bb = __ldg(Bp + i), cc = __ldg(Cp + i);
+            Bv[4 * i] = bb.x; Bv[4 * i + 1] = bb.y; Bv[4 * i + 2] = bb.z; Bv[4 * i + 3] = bb.w;
+            Cv[4 * i] = cc.x; Cv[4 * i + 1] = cc.y; Cv[4 * i + 2] = cc.z; Cv[4 * i + 3] = cc.w;
+        }
+    }
+    const float dtv = __ldg(p.dt + item);
+    const float Dv = p.D ? __ldg(p.D + h) : 0.0f;
+    float av[APS ? EPL : 1];
+    if constexpr (APS) {
+        const float4* Ap = reinterpret_cast<const float4*>(p.A + (size_t)h * N + n0);
+#pragma unroll
+        for (int i = 0; i < EPL / 4; ++i) {
+            const float4 aa = __ldg(Ap + i);
+            av[4 * i] = exp_spec(__fmul_rn(dtv, aa.x));
+            av[4 * i + 1] = exp_spec(__fmul_rn(dtv, aa.y));
+            av[4 * i + 2] = exp_spec(__fmul_rn(dtv, aa.z));
+            av[4 * i + 3] = exp_spec(__fmul_rn(dtv, aa.w));
+        }
+    } else {
+        av[0] = exp_spec(__fmul_rn(dtv, __ldg(p.A + h)));
+    }
+
+    LaneThreshold<FMT, RULE, LPR> thr;
+    thr.init(p.weyl, p.step_t, lis);
+    const uint32_t key0 = (uint32_t)p.sr_seed, key1 = (uint32_t)(p.sr_seed >> 32);
+
+    const uint32_t p_first = sub * p.rps;                         // first row of this slot inside the item
+    const uint64_t row_first = (uint64_t)item * p.P + p_first;    // local row index (this call's tensors)
+    const uint64_t grow_first = row_first + (uint64_t)p.batch_base * p.H * p.P;   // global row index
+    uint4* state = reinterpret_cast<uint4*>(p.state);
+    const bool row_scale = (FMT == FMT_E4M3) && (p.scale_block == (uint32_t)N);
+
+    float ykeep = 0.0f;
+    for (uint32_t k0 = 0; k0 < p.rps; k0 += UNR) {
+        uint4 raw[UNR];
+        float xv[UNR];
+        float sc[UNR];
+        bool ok[UNR];
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) {
+            const uint32_t k = k0 + u;
+            ok[u] = item_ok && (k < p.rps) && (p_first + k < p.P);
+            raw[u] = make_uint4(0u, 0u, 0u, 0u);
+            xv[u] = 0.0f;
+            sc[u] = 0.0f;
+            if (ok[u]) {
+                const uint64_t row = row_first + k;
+                raw[u] = state[row * LPR + lis];
+                xv[u] = __ldg(p.x + row);
+                if constexpr (FMT == FMT_E4M3)
+                    sc[u] = row_scale ? p.scales[row] : p.scales[row * (N / 16) + lis];
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) {
+            const uint32_t k = k0 + u;
+            const uint64_t row = row_first + k;
+            float hv[EPL];
+            unpack_lane<FMT>(raw[u], hv);
+            const float dtx = __fmul_rn(dtv, xv[u]);
+            float dot = 0.0f;
+            float amax = 0.0f;
+#pragma unroll
+            for (int j = 0; j < EPL; ++j) {
+                float hin = hv[j];
+                if constexpr (FMT == FMT_E4M3) hin = __fmul_rn(hin, sc[u]);
+                const float w = __fmul_rn(dtx, Bv[j]);
+                const float hn = __fmaf_rn(APS ? av[APS ? j : 0] : av[0], hin, w);
+                hv[j] = hn;
+                dot = __fmaf_rn(Cv[j], hn, dot);
+                if constexpr (FMT == FMT_E4M3) amax = fmaxf(amax, fabsf(hn));
+            }
+            // readout: reduce the partial dots over the slot
+#pragma unroll
+            for (int off = LPR / 2; off > 0; off >>= 1) dot += __shfl_xor_sync(FULL, dot, off);
+            if constexpr (FMT == FMT_E4M3) {
+                if (row_scale) {
+#pragma unroll
+                    for (int off = LPR / 2; off > 0; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, off));
+                }
+                const float s = fmaxf(__fdiv_rn(amax, 448.0f), 1.17549435e-38f);
+                const float rinv = __fdiv_rn(1.0f, s);
+#pragma unroll
+                for (int j = 0; j < EPL; ++j) hv[j] = __fmul_rn(hv[j], rinv);
+                if (ok[u]) {
+                    if (row_scale) { if (lis == 0) p.scales[row] = s; }
+                    else p.scales[row * (N / 16) + lis] = s;
+                }
+            }
+            uint32_t g_lo = 0, g_hi = 0, acc0 = 0;
+            if constexpr (RULE == RULE_WEYL) acc0 = thr.weyl_acc0(grow_first + k);
+            if constexpr (RULE == RULE_SR) thr.sr_group(grow_first + k, g_lo, g_hi);
+            const uint4 packed = round_pack_lane<FMT, RULE>(hv, acc0, p.weyl.mul_col, g_lo, g_hi, p.step_t, p.layer,
+                                                             key0, key1);
+            if (ok[u]) state[row * LPR + lis] = packed;
+            // y: lane (k mod LPR) of the slot keeps row k; flushed every LPR rows
+            const float yv = __fmaf_rn(Dv, xv[u], dot);
+            if ((k % LPR) == lis) ykeep = yv;
+            const bool last_of_batch = ((k % LPR) == LPR - 1) || (k + 1 == p.rps);
+            if (last_of_batch) {
+                const uint32_t kb = k - (k % LPR);                // first row of this batch of <= LPR rows
+                const uint32_t kk = kb + lis;
+                if (item_ok && kk <= k && kk < p.rps && (p_first + kk < p.P)) p.y[row_first + kk] = ykeep;
+            }
+        }
+    }
+}
+
+// Host-side launcher for one (format, rule): picks the lanes-per-row instantiation from N.
+template <int FMT, int RULE, int LPR, bool APS>
+inline cudaError_t launch_update_one(const UpdateParams& p, cudaStream_t stream) {
+    UpdateParams q = p;
+    const uint32_t nslot = kThreads / LPR;
+    uint32_t spi = 1;
+    while (spi < q.P && spi < nslot) spi <<= 1;        // slots per item: power of two, >= min(P, nslot)
+    q.spi = spi;
+    q.items_per_cta = nslot / spi;
+    q.rps = (q.P + spi - 1) / spi;
+    const uint32_t grid = (q.n_items + q.items_per_cta - 1) / q.items_per_cta;
+    ssd_update_kernel<FMT, RULE, LPR, APS><<<grid, kThreads, 0, stream>>>(q);
+    return cudaGetLastError();
+}
+
+template <int FMT, int RULE, bool APS>
+inline cudaError_t launch_update_n(const UpdateParams& p, cudaStream_t stream) {
+    constexpr int EPL = Fmt<FMT>::kEpl;
+    if (p.N % EPL != 0) return cudaErrorInvalidValue;
+    switch (p.N / EPL) {   // lanes per row; N = LPR * EPL must be one of 16, 32, 64, 128, 256 and LPR <= 32
+        case 1: if constexpr (EPL == 16) return launch_update_one<FMT, RULE, 1, APS>(p, stream); break;
+        case 2: if constexpr (EPL >= 8) return launch_update_one<FMT, RULE, 2, APS>(p, stream); break;
+        case 4: return launch_update_one<FMT, RULE, 4, APS>(p, stream);
+        case 8: return launch_update_one<FMT, RULE, 8, APS>(p, stream);
+        case 16: return launch_update_one<FMT, RULE, 16, APS>(p, stream);
+        case 32: if constexpr (EPL <= 8) return launch_update_one<FMT, RULE, 32, APS>(p, stream); break;
+        default: break;
+    }
+    return cudaErrorInvalidValue;
+}
+
+template <int FMT>
+inline cudaError_t launch_update_fmt(const UpdateParams& p, int rule, bool aps, cudaStream_t stream) {
+    if constexpr (FMT == FMT_FP32) {
+        return aps ? launch_update_n<FMT, RULE_RTN, true>(p, stream) : launch_update_n<FMT, RULE_RTN, false>(p, stream);
+    } else {
+        switch (rule) {
+            case RULE_RTN: return aps ? launch_update_n<FMT, RULE_RTN, true>(p, stream) : launch_update_n<FMT, RULE_RTN, false>(p, stream);
+            case RULE_SR: return aps ? launch_update_n<FMT, RULE_SR, true>(p, stream) : launch_update_n<FMT, RULE_SR, false>(p, stream);
+            case RULE_WEYL: return aps ? launch_update_n<FMT, RULE_WEYL, true>(p, stream) : launch_update_n<FMT, RULE_WEYL, false>(p, stream);
+            default: return cudaErrorInvalidValue;
+        }
+    }
+}
+
+}  // namespace ssdq

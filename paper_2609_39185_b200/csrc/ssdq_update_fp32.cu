@@ -1,0 +1,8 @@
+// Instantiations of the fused decode-step kernel for the fp32 state store.
+#include "ssdq_update.cuh"
+
+namespace ssdq {
+cudaError_t launch_update_fp32(const UpdateParams& p, int rule, bool a_per_state, cudaStream_t s) {
+    return launch_update_fmt<FMT_FP32>(p, rule, a_per_state, s);
+}
+}  // namespace ssdq

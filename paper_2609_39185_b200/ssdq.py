@@ -1,0 +1,171 @@
+"""ctypes binding of the C-ABI CUDA library (``include/ssdq.h``): argument marshalling only.
+
+Every function takes torch CUDA tensors (used as raw device pointers), enqueues the library's kernels
+on torch's current stream and returns without synchronising.  There is no fallback: if the compiled
+library is missing, or a call is rejected, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+FP16, BF16, E4M3, FP32 = 0, 1, 2, 3
+RTN, SR, WEYL = 0, 1, 2
+OK, ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_UNSUPPORTED, ERR_CUDA = 0, -1, -2, -3, -4, -5
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libssdq.so")
+
+EXPORTS = ("weyl_offsets_init", "ssdq_thresholds_materialize", "ssd_state_update", "quantize_store",
+           "ssdq_dequantize", "ssd_decode_run", "ssdq_last_error", "ssdq_launch_count")
+
+_u32, _u64, _i32, _vp = ctypes.c_uint32, ctypes.c_uint64, ctypes.c_int32, ctypes.c_void_p
+
+
+class SsdqError(RuntimeError):
+    def __init__(self, status, text):
+        super().__init__(f"ssdq status {status}: {text}")
+        self.status = status
+
+
+class Weyl(ctypes.Structure):
+    _fields_ = [("mul_row", _u32), ("mul_col", _u32), ("phi", _u32), ("base", _u32), ("block", _u32),
+                ("layer", _u32), ("seed", _u32), ("reserved", _u32)]
+
+
+class UpdateDesc(ctypes.Structure):
+    _fields_ = [("batch", _u32), ("nheads", _u32), ("headdim", _u32), ("dstate", _u32),
+                ("state", _vp), ("scales", _vp), ("scale_block", _u32), ("format", _i32),
+                ("x", _vp), ("dt", _vp), ("A", _vp), ("Bm", _vp), ("Cm", _vp), ("D", _vp),
+                ("a_per_state", _u32), ("y", _vp), ("rule", _i32), ("weyl", Weyl), ("sr_seed", _u64),
+                ("layer", _u32), ("batch_index_base", _u32)]
+
+
+class StepInputs(ctypes.Structure):
+    _fields_ = [("x", _vp), ("stride_x", _u64), ("dt", _vp), ("stride_dt", _u64), ("Bm", _vp), ("stride_B", _u64),
+                ("Cm", _vp), ("stride_C", _u64), ("y", _vp), ("stride_y", _u64), ("ring", _u32), ("reserved", _u32)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libssdq.so (built by ``python -m paper_2609_39185_b200.build``); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build the CUDA extension first "
+                              "(python -m paper_2609_39185_b200.build); there is no CPU fallback")
+        L = ctypes.CDLL(LIB_PATH)
+        L.weyl_offsets_init.restype = ctypes.c_int
+        L.weyl_offsets_init.argtypes = [ctypes.POINTER(Weyl), _u32, _u32, _u32]
+        L.ssdq_thresholds_materialize.restype = ctypes.c_int
+        L.ssdq_thresholds_materialize.argtypes = [ctypes.c_int, ctypes.POINTER(Weyl), _u64, _u32, _u64, _u64, _u32, _vp, _vp]
+        L.ssd_state_update.restype = ctypes.c_int
+        L.ssd_state_update.argtypes = [ctypes.POINTER(UpdateDesc), _u32, _vp]
+        L.quantize_store.restype = ctypes.c_int
+        L.quantize_store.argtypes = [_vp, _vp, _vp, _u64, _u32, _u32, ctypes.c_int, ctypes.c_int, ctypes.POINTER(Weyl),
+                                     _u64, _u32, _u64, _u32, _vp]
+        L.ssdq_dequantize.restype = ctypes.c_int
+        L.ssdq_dequantize.argtypes = [_vp, _vp, _u64, ctypes.c_int, _u32, _vp, _vp]
+        L.ssd_decode_run.restype = ctypes.c_int
+        L.ssd_decode_run.argtypes = [ctypes.POINTER(UpdateDesc), _u32, _u32, _u32, ctypes.POINTER(StepInputs), _vp]
+        L.ssdq_last_error.restype = ctypes.c_char_p
+        L.ssdq_last_error.argtypes = []
+        L.ssdq_launch_count.restype = _u64
+        L.ssdq_launch_count.argtypes = []
+        _lib = L
+    return _lib
+
+
+def _check(status):
+    if status != OK:
+        raise SsdqError(status, lib().ssdq_last_error().decode())
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def _stream():
+    import torch
+    return torch.cuda.current_stream().cuda_stream
+
+
+def weyl_offsets_init(layer: int = 0, seed: int = 0, block: int = 16) -> Weyl:
+    w = Weyl()
+    _check(lib().weyl_offsets_init(ctypes.byref(w), layer, seed, block))
+    return w
+
+
+def thresholds_materialize(rule, n, step_t, *, weyl=None, sr_seed=0, layer=0, first_flat=0):
+    """Test aid: the 24-bit thresholds of `n` consecutive entries as a CUDA uint32 tensor (as int32 storage)."""
+    import torch
+    out = torch.empty(n, dtype=torch.int32, device="cuda")
+    wp = ctypes.byref(weyl) if weyl is not None else None
+    _check(lib().ssdq_thresholds_materialize(rule, wp, sr_seed, layer, first_flat, n, step_t & 0xFFFFFFFF, _ptr(out), _stream()))
+    return out
+
+
+def make_desc(state, scales, fmt, *, A, D, rule, weyl=None, sr_seed=0, layer=0, scale_block=0, batch_index_base=0,
+              x=None, dt=None, Bm=None, Cm=None, y=None) -> UpdateDesc:
+    """Describe one layer's problem.  `state` is a CUDA tensor of shape [B, H, P, N] holding the codes
+    (uint8 for E4M3, int16/uint16/float16/bfloat16 for the 16-bit formats, float32 for the FP32 twin)."""
+    B, H, P, N = state.shape
+    d = UpdateDesc()
+    d.batch, d.nheads, d.headdim, d.dstate = B, H, P, N
+    d.state, d.scales, d.scale_block, d.format = _ptr(state), _ptr(scales), scale_block, fmt
+    d.x, d.dt, d.A, d.Bm, d.Cm, d.D = _ptr(x), _ptr(dt), _ptr(A), _ptr(Bm), _ptr(Cm), _ptr(D)
+    d.a_per_state = int(A.dim() == 2)
+    d.y = _ptr(y)
+    d.rule = rule
+    if weyl is not None:
+        d.weyl = weyl
+    d.sr_seed, d.layer, d.batch_index_base = sr_seed, layer, batch_index_base
+    # keep the tensors alive as long as the descriptor
+    d._keep = (state, scales, A, D, x, dt, Bm, Cm, y)
+    return d
+
+
+def ssd_state_update(desc: UpdateDesc, step_t: int, *, x=None, dt=None, Bm=None, Cm=None, y=None):
+    """One fused decode step of one layer, in place on desc.state; y is written.  Per-step tensors may be
+    given here (they overwrite the descriptor's pointers)."""
+    if x is not None:
+        desc.x, desc.dt, desc.Bm, desc.Cm, desc.y = _ptr(x), _ptr(dt), _ptr(Bm), _ptr(Cm), _ptr(y)
+    _check(lib().ssd_state_update(ctypes.byref(desc), step_t & 0xFFFFFFFF, _stream()))
+
+
+def quantize_store(src, codes, scales, fmt, rule, step_t, *, weyl=None, sr_seed=0, layer=0, scale_block=0,
+                   row_index_base=0):
+    """Quantise float32 CUDA tensor `src` [n_rows, row_len] into `codes` (and `scales` for E4M3)."""
+    n_rows, row_len = src.shape
+    wp = ctypes.byref(weyl) if weyl is not None else None
+    _check(lib().quantize_store(_ptr(src), _ptr(codes), _ptr(scales), n_rows, row_len, scale_block, fmt, rule, wp,
+                                sr_seed, layer, row_index_base, step_t & 0xFFFFFFFF, _stream()))
+
+
+def dequantize(codes, scales, fmt, out, scale_block=0):
+    _check(lib().ssdq_dequantize(_ptr(codes), _ptr(scales), codes.numel(), fmt, scale_block, _ptr(out), _stream()))
+
+
+def make_step_inputs(x, dt, Bm, Cm, y) -> StepInputs:
+    """x [ring, L, B, H, P], dt [ring, L, B, H], Bm/Cm [ring, L, B, N], y [ring, L, B, H, P] CUDA float32."""
+    s = StepInputs()
+    s.ring = x.shape[0]
+    s.x, s.stride_x = _ptr(x), x[0, 0].numel()
+    s.dt, s.stride_dt = _ptr(dt), dt[0, 0].numel()
+    s.Bm, s.stride_B = _ptr(Bm), Bm[0, 0].numel()
+    s.Cm, s.stride_C = _ptr(Cm), Cm[0, 0].numel()
+    s.y, s.stride_y = _ptr(y), y[0, 0].numel()
+    s._keep = (x, dt, Bm, Cm, y)
+    return s
+
+
+def ssd_decode_run(layer_descs, t_first: int, n_steps: int, step_inputs: StepInputs):
+    """n_steps decode steps over all layers on the current stream (one launch per layer per step)."""
+    arr = (UpdateDesc * len(layer_descs))(*layer_descs)
+    _check(lib().ssd_decode_run(arr, len(layer_descs), t_first & 0xFFFFFFFF, n_steps, ctypes.byref(step_inputs), _stream()))
+
+
+def launch_count() -> int:
+    return int(lib().ssdq_launch_count())

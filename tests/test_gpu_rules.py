@@ -1,0 +1,137 @@
+"""GPU parity of the rule machinery in isolation (through the C ABI): thresholds and quantize_store
+against the CPU oracle, bit for bit."""
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_39185_b200 import ssdq
+from parity import to_dev, codes_to_host, TORCH_CODE
+
+pytestmark = pytest.mark.gpu
+
+FMTS = [ssdq.FP16, ssdq.BF16, ssdq.E4M3]
+RULES = [ssdq.RTN, ssdq.SR, ssdq.WEYL]
+
+
+@pytest.mark.parametrize("first_flat", [0, 12345, 2**32 - 100, 2**36 + 3])
+@pytest.mark.parametrize("block", [16, 128])
+def test_weyl_thresholds_match_oracle(first_flat, block):
+    n = 5000
+    for layer, seed, t in ((0, 0, 1), (5, 1, 4096), (7, 3, 2**32 - 1)):
+        w = ssdq.weyl_offsets_init(layer, seed, block)
+        got = ssdq.thresholds_materialize(ssdq.WEYL, n, t, weyl=w, first_flat=first_flat).cpu().numpy().view(np.uint32)
+        want = oracle.thresholds(oracle.WEYL, range(first_flat, first_flat + n), t, layer=layer, weyl_seed=seed, weyl_block=block)
+        assert np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("first_flat", [0, 7, 2**34 + 1])
+def test_philox_thresholds_match_oracle(first_flat):
+    n = 4099
+    for layer, seed, t in ((0, 0, 1), (3, 0xDEADBEEFCAFE, 77)):
+        got = ssdq.thresholds_materialize(ssdq.SR, n, t, sr_seed=seed, layer=layer, first_flat=first_flat).cpu().numpy().view(np.uint32)
+        want = oracle.thresholds(oracle.SR, range(first_flat, first_flat + n), t, layer=layer, sr_seed=seed)
+        assert np.array_equal(got, want)
+
+
+def value_zoo(rng, n_rows, row_len, fmt):
+    """float32 rows that exercise every branch of Eq. 2 on the local grid: all binades of the format
+    including its subnormal range and values below it, exact grid points, zeros of both signs,
+    values beyond the largest finite number."""
+    lo, hi = {ssdq.FP16: (-50, 17), ssdq.BF16: (-126, 127), ssdq.E4M3: (-40, 10)}[fmt]
+    n = n_rows * row_len
+    e = rng.integers(lo, hi + 1, n)
+    m = rng.integers(0, 1 << 23, n).astype(np.uint32)
+    keep = {ssdq.FP16: 10, ssdq.BF16: 7, ssdq.E4M3: 3}[fmt]
+    m[::5] &= np.uint32(~((1 << (23 - keep)) - 1) & 0x7FFFFF)      # exact grid points (in the normal range)
+    m[1::11] = 0x7FFFFF                                             # just below a binade boundary
+    s = rng.integers(0, 2, n).astype(np.uint32)
+    bits = (s << 31) | ((e + 127).astype(np.uint32) << 23) | m
+    bits[2::97] = 0
+    bits[3::97] = 0x80000000
+    bits[4::97] = rng.integers(1, 1 << 23, len(bits[4::97])).astype(np.uint32)          # binary32 subnormals
+    bits[5::97] = 0x80000000 | rng.integers(1, 1 << 23, len(bits[5::97])).astype(np.uint32)
+    return bits.view(np.float32).reshape(n_rows, row_len)
+
+
+@pytest.mark.parametrize("fmt", FMTS)
+@pytest.mark.parametrize("rule", RULES)
+@pytest.mark.parametrize("row_len,weyl_block,scale_block", [(128, 128, 128), (128, 16, 16), (16, 16, 16), (64, 16, 64), (256, 16, 16), (32, 16, 32)])
+def test_quantize_store_matches_oracle(fmt, rule, row_len, weyl_block, scale_block):
+    rng = np.random.default_rng(1000 * fmt + 10 * rule + row_len)
+    n_rows = 700                                                    # not a multiple of the slots per CTA
+    src = value_zoo(rng, n_rows, row_len, fmt)
+    sb = scale_block if fmt == ssdq.E4M3 else 0
+    base, t, layer, seed = 2**30 + 5, 1234567, 4, 99
+    want_codes, want_scales = oracle.quantize_store(src, fmt, rule, t, scale_block=sb, layer=layer, weyl_seed=1,
+                                                    weyl_block=weyl_block, sr_seed=seed, row_index_base=base)
+    codes = torch.zeros((n_rows, row_len), dtype=TORCH_CODE[fmt], device="cuda")
+    scales = torch.zeros((n_rows, row_len // sb), dtype=torch.float32, device="cuda") if sb else None
+    w = ssdq.weyl_offsets_init(layer, 1, weyl_block)
+    ssdq.quantize_store(to_dev(src), codes, scales, fmt, rule, t, weyl=w, sr_seed=seed, layer=layer, scale_block=sb,
+                        row_index_base=base)
+    torch.cuda.synchronize()
+    got = codes_to_host(codes, fmt)
+    bad = np.argwhere(got != want_codes)
+    assert len(bad) == 0, (len(bad), src[tuple(bad[0])].item().hex(), hex(int(got[tuple(bad[0])])), hex(int(want_codes[tuple(bad[0])])))
+    if sb:
+        assert np.array_equal(scales.cpu().numpy().view(np.uint32), want_scales.view(np.uint32))
+
+
+@pytest.mark.parametrize("fmt", [ssdq.FP16, ssdq.E4M3])
+def test_subnormal_decision_boundary(fmt):
+    """Values below the format's normal range whose kept bits sit exactly on the round-up boundary:
+    the dropped low bits of the value and of the threshold decide.  Thresholds are steered by solving
+    the Weyl accumulator for the write index t (Phi is odd, hence invertible modulo 2^32)."""
+    mant, emin = {ssdq.FP16: (10, -14), ssdq.E4M3: (3, -6)}[fmt]
+    drop = 23 - mant
+    phi_inv = pow(2654435769, -1, 2**32)
+    w = ssdq.weyl_offsets_init(0, 0, 16)
+    rng = np.random.default_rng(7 + fmt)
+    row_len, n_rows = 16, 64
+    for trial in range(24):
+        # one write index t per trial; entry (0, 0) is steered onto the boundary, the rest is a zoo
+        e = int(rng.integers(emin - 30, emin))                     # subnormal target
+        mbits = int(rng.integers(0, 1 << 23))
+        sign = int(rng.integers(0, 2))
+        v = np.uint32((sign << 31) | ((e + 127) << 23) | mbits).view(np.float32)
+        # kept fraction bits F of |v| on the first binade: mantissa of |v| + 2^emin, truncated
+        F = int(Fraction(abs(float(v))) / Fraction(2) ** (emin - 23)) & ((1 << drop) - 1)
+        r_needed = ((1 << drop) - 1) - F                           # F + r == all ones
+        low = int(rng.integers(0, 1 << (32 - drop)))
+        acc_top = r_needed if sign == 0 else ((1 << drop) - 1) - r_needed
+        target_acc = ((acc_top << (32 - drop)) | low) & 0xFFFFFFFF
+        # acc(r=0, c=0, t) = mul_row + mul_col + base + t*phi  =>  t
+        t = ((target_acc - (w.mul_row + w.mul_col + w.base)) * phi_inv) % 2**32
+        src = value_zoo(rng, n_rows, row_len, fmt)
+        src[0, 0] = v
+        sb = 16 if fmt == ssdq.E4M3 else 0
+        if fmt == ssdq.E4M3:
+            src[0, 1:] = 0.0
+            src[0, 1] = 448.0          # block scale exactly 1: the steered value reaches the rounding unchanged
+        want_codes, _ = oracle.quantize_store(src, fmt, ssdq.WEYL, t, scale_block=sb, weyl_block=16)
+        codes = torch.zeros((n_rows, row_len), dtype=TORCH_CODE[fmt], device="cuda")
+        scales = torch.zeros((n_rows, 1), dtype=torch.float32, device="cuda") if sb else None
+        ssdq.quantize_store(to_dev(src), codes, scales, fmt, ssdq.WEYL, t, weyl=w, scale_block=sb)
+        torch.cuda.synchronize()
+        assert np.array_equal(codes_to_host(codes, fmt), want_codes), trial
+
+
+@pytest.mark.parametrize("fmt", FMTS + [ssdq.FP32])
+def test_dequantize_matches_oracle(fmt):
+    rng = np.random.default_rng(3)
+    n_rows, row_len = 33, 128
+    sb = 128 if fmt == ssdq.E4M3 else 0
+    if fmt == ssdq.FP32:
+        codes_h = rng.standard_normal((n_rows, row_len)).astype(np.float32).view(np.uint32)
+        scales_h = None
+    else:
+        codes_h, scales_h = oracle.quantize_store(rng.standard_normal((n_rows, row_len)).astype(np.float32) * 3, fmt,
+                                                  oracle.RTN, 1, scale_block=sb)
+    from parity import codes_to_dev
+    out = torch.empty((n_rows, row_len), dtype=torch.float32, device="cuda")
+    ssdq.dequantize(codes_to_dev(codes_h, fmt), to_dev(scales_h), fmt, out, scale_block=sb)
+    want = oracle.dequantize(codes_h, scales_h, fmt, sb)
+    assert np.array_equal(out.cpu().numpy().view(np.uint32), want.view(np.uint32))

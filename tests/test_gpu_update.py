@@ -1,0 +1,207 @@
+"""GPU parity of the fused decode step (through the C ABI) against the CPU oracle: stored state bit
+for bit, y within 1e-5 of the absolute-sum scale, on the five named workloads and on edge shapes."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_39185_b200 import ssdq, workloads
+from parity import Pair, run_parity, to_dev, codes_to_dev, codes_to_host
+
+pytestmark = pytest.mark.gpu
+
+RULES = [ssdq.RTN, ssdq.SR, ssdq.WEYL]
+CFG = workloads.CONFIGS
+
+
+@pytest.mark.parametrize("rule", RULES)
+def test_config1_tiny_fp16_full_horizon(rule):
+    run_parity(CFG[1], rule, CFG[1].steps)
+
+
+@pytest.mark.parametrize("rule", RULES)
+def test_config2_mamba1_bf16_full_horizon(rule):
+    run_parity(CFG[2], rule, CFG[2].steps, check_every=16)
+
+
+@pytest.mark.parametrize("rule", RULES)
+def test_config3_mamba2_fp16_full_size_few_steps(rule):
+    run_parity(CFG[3], rule, 3)
+
+
+@pytest.mark.parametrize("rule", RULES)
+def test_config3_full_horizon_on_a_batch_slice(rule):
+    # sequences are independent: the last two sequences, addressed with their global batch index
+    run_parity(CFG[3], rule, CFG[3].steps, batch_slice=slice(62, 64), batch_index_base=62, check_every=32)
+
+
+@pytest.mark.parametrize("rule", RULES)
+def test_config4_e4m3_full_size_few_steps(rule):
+    run_parity(CFG[4], rule, 4)
+
+
+@pytest.mark.parametrize("rule", RULES)
+def test_config4_long_horizon_on_one_sequence(rule):
+    run_parity(CFG[4], rule, 768, batch_slice=slice(31, 32), batch_index_base=31, check_every=64)
+
+
+@pytest.mark.parametrize("rule", RULES)
+def test_config5_full_batch_launch_sampled_sequences(rule):
+    """The launch configuration the benchmark times (B=128, H=128, P=64, N=128, bf16), two layers with
+    their own seeds, a few steps; the oracle recomputes sequences 0, 1, 126, 127."""
+    cfg = CFG[5]
+    steps = 3
+    for layer in (0, 7):
+        seed = workloads.layer_seed(cfg, 0, layer)
+        A, D = workloads.layer_params(cfg, layer, seed)
+        gpu = Pair(cfg.state_shape, cfg.fmt, rule, A, D, weyl_block=cfg.weyl_block, layer=layer, sr_seed=seed)
+        subs = {0: Pair((2,) + cfg.state_shape[1:], cfg.fmt, rule, A, D, weyl_block=cfg.weyl_block, layer=layer,
+                        sr_seed=seed, batch_index_base=0),
+                126: Pair((2,) + cfg.state_shape[1:], cfg.fmt, rule, A, D, weyl_block=cfg.weyl_block, layer=layer,
+                          sr_seed=seed, batch_index_base=126)}
+        for t in range(1, steps + 1):
+            x, dt, Bm, Cm = workloads.step_inputs(cfg, t, layer, seed)
+            y = gpu.step_gpu(t, x, dt, Bm, Cm).cpu().numpy()
+            got = codes_to_host(gpu.state_d, cfg.fmt)
+            for b0, sub in subs.items():
+                sl = slice(b0, b0 + 2)
+                y_ref = sub.step_oracle(t, x[sl], dt[sl], Bm[sl], Cm[sl])
+                assert np.array_equal(got[sl], sub.state_h), (layer, t, b0)
+                new_f32 = oracle.dequantize(sub.state_h, None, cfg.fmt).reshape(sub.shape)
+                from parity import y_close
+                ok, worst = y_close(y[sl], y_ref, Cm[sl], new_f32, D, x[sl])
+                assert ok, (layer, t, b0, worst)
+        del gpu
+        torch.cuda.empty_cache()
+
+
+SHAPES = [
+    # (B, H, P, N, a_per_state)
+    (1, 1, 1, 16, False), (3, 5, 7, 16, True), (2, 3, 64, 128, False), (5, 7, 3, 128, False), (2, 2, 100, 64, False),
+    (1, 9, 8, 256, False), (2, 130, 1, 32, True), (1, 3, 65, 128, True), (4, 1, 16, 64, True),
+]
+
+
+@pytest.mark.parametrize("fmt", [ssdq.FP16, ssdq.BF16, ssdq.E4M3, ssdq.FP32])
+@pytest.mark.parametrize("rule", RULES)
+@pytest.mark.parametrize("shape", SHAPES)
+def test_edge_shapes_and_options(fmt, rule, shape):
+    B, H, P, N, aps = shape
+    if fmt == ssdq.FP32 and (N > 128 or rule != ssdq.RTN):
+        pytest.skip("the FP32 twin never rounds and is built for N <= 128")
+    rng = np.random.default_rng(hash((fmt, rule) + shape) % 2**32)
+    f32 = np.float32
+    A = -np.exp(rng.uniform(-4, 1, (H, N) if aps else (H,))).astype(f32)
+    use_D = (B + H) % 2 == 0
+    D = rng.normal(0, 0.1, H).astype(f32) if use_D else None
+    wb = 16 if (P + N) % 3 else N
+    sb = 0
+    if fmt == ssdq.E4M3:
+        sb = 16 if P % 2 else N
+    src = (rng.standard_normal((B * H * P, N)) * 0.3).astype(f32)
+    base = 11
+    if fmt == ssdq.FP32:
+        h0 = (src.view(np.uint32).copy(), None)
+    else:
+        h0 = oracle.quantize_store(src, fmt, oracle.RTN, 1, scale_block=sb, weyl_block=wb)
+    pair = Pair((B, H, P, N), fmt, rule, A, D, weyl_block=wb, scale_block=sb, layer=3, weyl_seed=2, sr_seed=12345,
+                batch_index_base=base, h0_codes=h0[0], h0_scales=h0[1])
+    for t in range(2, 6):
+        x = rng.standard_normal((B, H, P)).astype(f32)
+        dt = np.log1p(np.exp(rng.normal(-2, 1, (B, H)))).astype(f32)
+        Bm = rng.standard_normal((B, N)).astype(f32)
+        Cm = rng.standard_normal((B, N)).astype(f32)
+        pair.step_gpu(t, x, dt, Bm, Cm)
+        y_ref = pair.step_oracle(t, x, dt, Bm, Cm)
+        pair.compare(t, x, dt, Bm, Cm, y_ref)
+
+
+@pytest.mark.parametrize("fmt", [ssdq.FP16, ssdq.BF16, ssdq.E4M3])
+def test_extreme_values_saturate_and_keep_signed_zero(fmt):
+    """Decay to (sub)normal dust, growth beyond the largest finite value, exact zeros of both signs."""
+    rng = np.random.default_rng(5)
+    B, H, P, N = 1, 4, 4, 128
+    f32 = np.float32
+    A = np.array([-40.0, -1e-6, -3.0, 0.0], f32)           # fast decay / almost none / medium / a = 1
+    sb = N if fmt == ssdq.E4M3 else 0
+    for rule in RULES:
+        pair = Pair((B, H, P, N), fmt, rule, A, None, weyl_block=N, scale_block=sb)
+        for t in range(1, 40):
+            big = (t % 7 == 3)
+            x = (rng.standard_normal((B, H, P)) * (1e6 if big else 1.0)).astype(f32)
+            if t % 5 == 0:
+                x[:] = 0.0
+            if t % 5 == 1:
+                x[:] = -0.0
+            dt = np.full((B, H), 2.0, f32)
+            Bm = (rng.standard_normal((B, N)) * (1e3 if big else 1e-3)).astype(f32)
+            Cm = rng.standard_normal((B, N)).astype(f32)
+            pair.step_gpu(t, x, dt, Bm, Cm)
+            y_ref = pair.step_oracle(t, x, dt, Bm, Cm)
+            pair.compare(t, x, dt, Bm, Cm, y_ref, y_rel_to_max=1e-5)
+
+
+def test_decode_driver_equals_repeated_updates_and_resumes():
+    """ssd_decode_run over a ring of inputs == one ssd_state_update per (step, layer); and because every
+    rule is a function of (index, t, seed) only, stopping and resuming reproduces the same bits."""
+    cfg = workloads.CONFIGS[1].with_batch(3)
+    L, T = 2, 12
+    for rule in RULES:
+        params = [workloads.layer_params(cfg, l, l) for l in range(L)]
+        ins = [[workloads.step_inputs(cfg, t, l, l) for l in range(L)] for t in range(1, T + 1)]
+        stack = lambda i: to_dev(np.stack([np.stack([ins[t][l][i] for l in range(L)]) for t in range(T)]))
+        xs, dts, Bs, Cs = (stack(i) for i in range(4))
+        ys = torch.zeros_like(xs)
+
+        def fresh():
+            states = [torch.zeros(cfg.state_shape, dtype=torch.int16, device="cuda") for _ in range(L)]
+            descs = [ssdq.make_desc(states[l], None, cfg.fmt, A=to_dev(params[l][0]), D=to_dev(params[l][1]), rule=rule,
+                                    weyl=ssdq.weyl_offsets_init(l, 0, cfg.weyl_block), sr_seed=l, layer=l) for l in range(L)]
+            return states, descs
+
+        s1, d1 = fresh()
+        ssdq.ssd_decode_run(d1, 1, T, ssdq.make_step_inputs(xs, dts, Bs, Cs, ys))
+        s2, d2 = fresh()
+        y2 = torch.zeros_like(ys)
+        for t in range(T):
+            for l in range(L):
+                ssdq.ssd_state_update(d2[l], t + 1, x=xs[t, l], dt=dts[t, l], Bm=Bs[t, l], Cm=Cs[t, l], y=y2[t, l])
+        s3, d3 = fresh()
+        y3 = torch.zeros_like(ys)
+        ssdq.ssd_decode_run(d3, 1, 5, ssdq.make_step_inputs(xs[:5], dts[:5], Bs[:5], Cs[:5], y3[:5]))
+        torch.cuda.synchronize()
+        saved = [s.clone() for s in s3]                       # "checkpoint": the codes are the whole state
+        s4, d4 = fresh()
+        for l in range(L):
+            s4[l].copy_(saved[l])
+        ssdq.ssd_decode_run(d4, 6, T - 5, ssdq.make_step_inputs(xs[5:], dts[5:], Bs[5:], Cs[5:], y3[5:]))
+        torch.cuda.synchronize()
+        for l in range(L):
+            assert torch.equal(s1[l], s2[l]) and torch.equal(s1[l], s4[l])
+        assert torch.equal(ys, y2) and torch.equal(ys, y3)
+        # and the oracle agrees on the final state
+        for l in range(L):
+            st, _ = oracle.new_state(cfg.state_shape, cfg.fmt)
+            for t in range(T):
+                oracle.state_update(st, None, cfg.fmt, 0, *ins[t][l][:2], params[l][0], *ins[t][l][2:], params[l][1], rule,
+                                    t + 1, layer=l, weyl_block=cfg.weyl_block, sr_seed=l)
+            assert np.array_equal(codes_to_host(s1[l], cfg.fmt), st)
+
+
+def test_ring_reuses_inputs():
+    cfg = workloads.CONFIGS[1]
+    A, D = workloads.layer_params(cfg)
+    ring, T = 3, 7
+    ins = [workloads.step_inputs(cfg, t) for t in range(1, ring + 1)]
+    stack = lambda i: to_dev(np.stack([ins[t][i][None] for t in range(ring)]))
+    xs, dts, Bs, Cs = (stack(i) for i in range(4))
+    ys = torch.zeros_like(xs)
+    state = torch.zeros(cfg.state_shape, dtype=torch.int16, device="cuda")
+    desc = ssdq.make_desc(state, None, cfg.fmt, A=to_dev(A), D=to_dev(D), rule=ssdq.WEYL, weyl=ssdq.weyl_offsets_init(0, 0, 16))
+    ssdq.ssd_decode_run([desc], 1, T, ssdq.make_step_inputs(xs, dts, Bs, Cs, ys))
+    st, _ = oracle.new_state(cfg.state_shape, cfg.fmt)
+    for i in range(T):
+        x, dt, Bm, Cm = ins[i % ring]
+        oracle.state_update(st, None, cfg.fmt, 0, x, dt, A, Bm, Cm, D, oracle.WEYL, 1 + i, weyl_block=16)
+    torch.cuda.synchronize()
+    assert np.array_equal(codes_to_host(state, cfg.fmt), st)
