@@ -1,0 +1,347 @@
+#!/usr/bin/env python
+"""Benchmark of the fused quantized state-update decode step on one B200 (or N independent replicas).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--rule weyl|rtn|sr] [--config 5] [--impl reference]
+
+A "step" is one decode step of the whole hot path over one batch: every layer of the configuration
+is updated once (one fused kernel launch per layer).  The default workload is configuration 5, the
+hybrid-model-shaped stack (8 layers x [B=128, H=128, P=64, N=128] BF16 state, 2.1 GB: far beyond L2,
+so no L2 flush is needed between steps).  The headline value is algorithmic state-update bandwidth:
+bytes the method must move per step / device time per step.
+
+Prints ONE JSON line.  `--impl reference` times the CPU oracle instead (the reported CPU baseline).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2609_39185_b200 import workloads  # noqa: E402
+
+RULE_IDS = {"rtn": 0, "sr": 1, "weyl": 2}
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured (MEASURED_PEAKS.json, stream copy)"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback (earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm = [float(r[0]) for r in self.rows if r and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) > 1 and r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(len(r) > 3 + i and r[3 + i] == "Active" for r in self.rows)]
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(sm)}
+
+
+def make_ring(cfg, ring, seed, pin=False):
+    """Host arrays of `ring` decode steps for every layer: x [R,L,B,H,P], dt [R,L,B,H], Bm, Cm [R,L,B,N]."""
+    import torch
+    L = cfg.n_layers
+    B, H, P, N = cfg.state_shape
+    xs = torch.empty((ring, L, B, H, P), dtype=torch.float32, pin_memory=pin)
+    dts = torch.empty((ring, L, B, H), dtype=torch.float32, pin_memory=pin)
+    Bs = torch.empty((ring, L, B, N), dtype=torch.float32, pin_memory=pin)
+    Cs = torch.empty((ring, L, B, N), dtype=torch.float32, pin_memory=pin)
+    for r in range(ring):
+        for l in range(L):
+            x, dt, Bm, Cm = workloads.step_inputs(cfg, r + 1, l, workloads.layer_seed(cfg, seed, l))
+            xs[r, l], dts[r, l], Bs[r, l], Cs[r, l] = (torch.from_numpy(v) for v in (x, dt, Bm, Cm))
+    return xs, dts, Bs, Cs
+
+
+class Stack:
+    """All layers of one configuration resident on the current GPU."""
+
+    def __init__(self, cfg, rule, seed=0, batch_index_base=0):
+        import torch
+        from paper_2609_39185_b200 import ssdq
+        self.cfg, self.rule, self.ssdq = cfg, rule, ssdq
+        code_dtype = torch.uint8 if cfg.fmt == workloads.E4M3 else torch.int16
+        self.states, self.scales, self.descs, self.keep = [], [], [], []
+        for l in range(cfg.n_layers):
+            ls = workloads.layer_seed(cfg, seed, l)
+            A, D = workloads.layer_params(cfg, l, ls)
+            A_d, D_d = torch.from_numpy(A).cuda(), torch.from_numpy(D).cuda()
+            st = torch.zeros(cfg.state_shape, dtype=code_dtype, device="cuda")
+            sc = None
+            if cfg.fmt == workloads.E4M3:
+                sc = torch.full((cfg.entries_per_layer // cfg.scale_block,), float(np.finfo(np.float32).tiny),
+                                dtype=torch.float32, device="cuda")
+            w = ssdq.weyl_offsets_init(l, 0, cfg.weyl_block)
+            self.descs.append(ssdq.make_desc(st, sc, cfg.fmt, A=A_d, D=D_d, rule=rule, weyl=w, sr_seed=ls, layer=l,
+                                             scale_block=cfg.scale_block, batch_index_base=batch_index_base))
+            self.states.append(st)
+            self.scales.append(sc)
+
+    def set_rule(self, rule):
+        for d in self.descs:
+            d.rule = rule
+
+    def run(self, t_first, n_steps, step_inputs):
+        self.ssdq.ssd_decode_run(self.descs, t_first, n_steps, step_inputs)
+
+
+def time_steps(stack, step_inputs, t_first, n_steps):
+    """Device time of n_steps decode steps, CUDA events on the launching (current) stream."""
+    import torch
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    stack.run(t_first, n_steps, step_inputs)
+    e1.record()
+    e1.synchronize()
+    return e0.elapsed_time(e1) / 1e3
+
+
+def oracle_sample(cfg, rule, seed=0, target_seconds=12.0):
+    """The CPU oracle, as it stands, on a bounded sample of the same workload: a slice of the batch of
+    every layer, decoded for a few steps on the host cores.  Returns (GB/s, steps/s at full batch, info)."""
+    import oracle
+    nb = min(cfg.batch, 8)
+    sub = cfg.with_batch(nb)
+    per_layer = []
+    for l in range(cfg.n_layers):
+        ls = workloads.layer_seed(cfg, seed, l)
+        A, D = workloads.layer_params(cfg, l, ls)
+        st, sc = oracle.new_state(sub.state_shape, cfg.fmt, cfg.scale_block)
+        per_layer.append((ls, A, D, st, sc))
+    ins = {l: workloads.step_inputs(cfg, 1, l, per_layer[l][0], slice(0, nb)) for l in range(cfg.n_layers)}
+    oracle.lib()
+    t0 = time.perf_counter()
+    steps = 0
+    while True:
+        for l, (ls, A, D, st, sc) in enumerate(per_layer):
+            x, dt, Bm, Cm = ins[l]
+            oracle.state_update(st, sc, cfg.fmt, cfg.scale_block, x, dt, A, Bm, Cm, D, rule, steps + 1, layer=l,
+                                weyl_block=cfg.weyl_block, sr_seed=ls)
+        steps += 1
+        el = time.perf_counter() - t0
+        if el > target_seconds or steps >= 64:
+            break
+    bytes_per_step = sub.algorithmic_bytes_per_layer_step() * cfg.n_layers
+    gbs = bytes_per_step * steps / el / 1e9
+    full_steps_per_s = steps / el * nb / cfg.batch
+    info = f"{steps} steps of {cfg.n_layers} layers on sequences 0..{nb - 1} of {cfg.batch} ({el:.1f} s)"
+    return gbs, full_steps_per_s, oracle.num_threads(), info
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    gbs, sps, cores, info = oracle_sample(cfg, RULE_IDS[args.rule], target_seconds=max(4.0, 3.0 * args.steps))
+    line = {"impl": "reference", "metric": "state_update_hbm_gbs", "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 / sps if sps else None,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": workload_config(cfg, args),
+            "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": info},
+            "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def workload_config(cfg, args):
+    B, H, P, N = cfg.state_shape
+    return {"workload": f"config {cfg.index}: {cfg.name}", "layers": cfg.n_layers, "batch": B, "nheads": H,
+            "headdim": P, "dstate": N, "state_format": workloads.FORMAT_NAMES[cfg.fmt], "rule": args.rule,
+            "state_bytes": cfg.state_bytes_per_layer() * cfg.n_layers, "ring_steps": args.ring,
+            "l2": "state larger than L2 (no flush needed)" if cfg.state_bytes_per_layer() * cfg.n_layers > 256e6
+                  else "state may be L2-resident",
+            "parallelism": f"replicas x{args.gpus} (batch shards, no collective)"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--rule", default="weyl", choices=list(RULE_IDS))
+    ap.add_argument("--config", type=int, default=5)
+    ap.add_argument("--batch", type=int, default=0, help="override the configuration's batch")
+    ap.add_argument("--ring", type=int, default=4, help="distinct decode steps of inputs kept resident")
+    ap.add_argument("--no-extras", action="store_true", help="skip the per-rule sweep, e2e and CPU baseline")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    cfg = workloads.CONFIGS[args.config]
+    if args.batch:
+        cfg = cfg.with_batch(args.batch)
+    if args.impl == "reference":
+        return run_reference(args, cfg)
+
+    import torch
+    from paper_2609_39185_b200 import ssdq
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    rule = RULE_IDS[args.rule]
+    stack = Stack(cfg, rule, batch_index_base=rank * cfg.batch)
+    xs_h, dts_h, Bs_h, Cs_h = make_ring(cfg, args.ring, 0, pin=True)
+    xs, dts, Bs, Cs = (t.cuda() for t in (xs_h, dts_h, Bs_h, Cs_h))
+    ys = torch.empty_like(xs)
+    sin = ssdq.make_step_inputs(xs, dts, Bs, Cs, ys)
+    bytes_per_launch = cfg.algorithmic_bytes_per_layer_step()
+    bytes_per_step = bytes_per_launch * cfg.n_layers
+
+    # ---- device-resident timing: W warm-up steps, then exactly K steps ----
+    stack.run(1, args.warmup, sin)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = ssdq.launch_count()
+    barrier()
+    secs = time_steps(stack, sin, 1 + args.warmup, args.steps)
+    barrier()
+    launches = ssdq.launch_count() - launches0
+    clocks = sampler.stop()
+    if dist is not None:
+        tt = torch.tensor([secs], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        secs = float(tt.item())
+    gbs = bytes_per_step * args.steps * world / secs / 1e9
+    launch_secs = secs / (args.steps * cfg.n_layers)
+    peak, peak_src = measured_peak()
+    achieved = bytes_per_launch / launch_secs / 1e9
+
+    line = {"metric": "state_update_hbm_gbs", "value": gbs, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": secs / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(cfg, args),
+            "steps_per_s": args.steps / secs, "pct_of_nominal_8tbs": 100.0 * gbs / world / NOMINAL_HBM_GBS,
+            "pct_of_measured_copy": 100.0 * gbs / world / peak,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": None, "kernel": "ssd_update_kernel", "peak_source": peak_src,
+                         "algorithmic_bytes_per_launch": bytes_per_launch, "launch_us": launch_secs * 1e6},
+            "clocks": clocks, "gpu_launches": int(launches)}
+
+    if not args.no_extras:
+        # ---- per-rule sweep: interleaved rounds over {copy, rtn, sr, weyl}, median per rule ----
+        rounds, reps = 7, max(10, min(50, args.steps))
+        times = {k: [] for k in ("copy", "rtn", "sr", "weyl")}
+        dst = torch.empty_like(stack.states[0])
+        for _ in range(rounds):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                for st in stack.states:
+                    dst.copy_(st)
+            e1.record()
+            e1.synchronize()
+            times["copy"].append(e0.elapsed_time(e1) / 1e3 / reps)
+            for name, rid in RULE_IDS.items():
+                stack.set_rule(rid)
+                times[name].append(time_steps(stack, sin, 1, reps) / reps)
+        stack.set_rule(rule)
+        copy_bytes = 2 * cfg.state_bytes_per_layer() * cfg.n_layers
+        med = {k: float(np.median(v)) for k, v in times.items()}
+        line["rules"] = {k: {"ms_per_step": med[k] * 1e3,
+                             "gbs": (copy_bytes if k == "copy" else bytes_per_step) / med[k] / 1e9} for k in med}
+        line["weyl_over_rtn_time"] = med["weyl"] / med["rtn"]
+        line["sr_over_rtn_time"] = med["sr"] / med["rtn"]
+
+        # ---- end to end: per step, inputs come from pinned host memory and y goes back to the host ----
+        in_bytes = sum(t[0].numel() * 4 for t in (xs_h, dts_h, Bs_h, Cs_h))
+        out_bytes = ys[0].numel() * 4
+        ys_h = torch.empty(ys[0].shape, dtype=torch.float32, pin_memory=True)
+        one = ssdq.make_step_inputs(xs[:1], dts[:1], Bs[:1], Cs[:1], ys[:1])
+        e2e_steps = max(3, min(args.steps, 50))
+
+        def e2e_step(i):
+            r = i % args.ring
+            xs[0].copy_(xs_h[r], non_blocking=True)
+            dts[0].copy_(dts_h[r], non_blocking=True)
+            Bs[0].copy_(Bs_h[r], non_blocking=True)
+            Cs[0].copy_(Cs_h[r], non_blocking=True)
+            stack.run(1 + i, 1, one)
+            ys_h.copy_(ys[0], non_blocking=True)
+
+        for i in range(3):
+            e2e_step(i)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(e2e_steps):
+            e2e_step(i)
+        e1.record()
+        e1.synchronize()
+        e2e_secs = e0.elapsed_time(e1) / 1e3
+        if dist is not None:
+            tt = torch.tensor([e2e_secs], device="cuda", dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            e2e_secs = float(tt.item())
+        line["e2e"] = {"value": bytes_per_step * e2e_steps * world / e2e_secs / 1e9, "unit": "GB/s",
+                       "h2d_bytes_per_step": int(in_bytes), "d2h_bytes_per_step": int(out_bytes),
+                       "ms_per_step": e2e_secs / e2e_steps * 1e3, "steps": e2e_steps,
+                       "note": "state stays resident in HBM; per-step inputs from pinned host memory, y back to host"}
+
+        # ---- CPU baseline: the oracle on the host cores, rank 0 at N=1 only ----
+        if world == 1:
+            cgbs, csps, cores, info = oracle_sample(cfg, rule)
+            line["cpu_baseline"] = {"value": cgbs, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": info,
+                                    "steps_per_s_full_batch": csps}
+    barrier()
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
