@@ -203,6 +203,7 @@ def main():
     ap.add_argument("--rule", default="weyl", choices=list(RULE_IDS))
     ap.add_argument("--config", type=int, default=5)
     ap.add_argument("--batch", type=int, default=0, help="override the configuration's batch")
+    ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling captures)")
     ap.add_argument("--ring", type=int, default=4, help="distinct decode steps of inputs kept resident")
     ap.add_argument("--no-extras", action="store_true", help="skip the per-rule sweep, e2e and CPU baseline")
     args = ap.parse_args()
@@ -211,6 +212,9 @@ def main():
     cfg = workloads.CONFIGS[args.config]
     if args.batch:
         cfg = cfg.with_batch(args.batch)
+    if args.layers:
+        from dataclasses import replace
+        cfg = replace(cfg, n_layers=args.layers)
     if args.impl == "reference":
         return run_reference(args, cfg)
 

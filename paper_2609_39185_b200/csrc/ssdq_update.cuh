@@ -76,20 +76,46 @@ __device__ __forceinline__ uint4 round_pack_lane(const float* v, uint32_t acc0, 
                 acc[4 * g] = o.x; acc[4 * g + 1] = o.y; acc[4 * g + 2] = o.z; acc[4 * g + 3] = o.w;
             }
         }
-        if constexpr (FMT == FMT_FP16) {
+        if constexpr (FMT == FMT_BF16) {
+            uint32_t any = 0;
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                w[i] = dither_code_fp16(v[2 * i], acc[2 * i]) | (dither_code_fp16(v[2 * i + 1], acc[2 * i + 1]) << 16);
-        } else if constexpr (FMT == FMT_BF16) {
+            for (int i = 0; i < 4; ++i) {
+                w[i] = trunc_pack2_bf16(dither_sum_bf16(v[2 * i], acc[2 * i]), dither_sum_bf16(v[2 * i + 1], acc[2 * i + 1]));
+                any |= w[i];
+            }
+            if (any & 0x40004000u) {   // some |code| >= 2: it may sit at the top of the range, take the clamped route
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                w[i] = dither_code_bf16(v[2 * i], acc[2 * i]) | (dither_code_bf16(v[2 * i + 1], acc[2 * i + 1]) << 16);
+                for (int i = 0; i < 4; ++i)
+                    w[i] = dither_code_bf16_clamped(v[2 * i], acc[2 * i]) | (dither_code_bf16_clamped(v[2 * i + 1], acc[2 * i + 1]) << 16);
+            }
+        } else if constexpr (FMT == FMT_FP16) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                float r[2];
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    const float vv = v[2 * i + j];
+                    const float scale = dither_step_scale<10, -14, 24>(vv);
+                    const float q = floor_to_step(dithered_sum_rm(vv, acc[2 * i + j], scale), scale);
+                    // sign of v forced onto the result (it already has it unless it is zero)
+                    r[j] = __uint_as_float((__float_as_uint(q) & 0x7FFFFFFFu) | (__float_as_uint(vv) & 0x80000000u));
+                }
+                w[i] = rtn_pack2_fp16(r[0], r[1]);   // exact: r is on the FP16 grid; saturates beyond 65504
+            }
         } else {
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                w[i] = dither_code_e4m3(v[4 * i], acc[4 * i]) | (dither_code_e4m3(v[4 * i + 1], acc[4 * i + 1]) << 8) |
-                       (dither_code_e4m3(v[4 * i + 2], acc[4 * i + 2]) << 16) |
-                       (dither_code_e4m3(v[4 * i + 3], acc[4 * i + 3]) << 24);
+            for (int i = 0; i < 4; ++i) {
+                float r[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float vv = v[4 * i + j];
+                    const float scale = dither_step_scale<3, -6, 127>(vv);
+                    const float q = floor_to_step(dithered_sum_rm(vv, acc[4 * i + j], scale), scale);
+                    // sign of v forced onto the result (it already has it unless it is zero)
+                    r[j] = __uint_as_float((__float_as_uint(q) & 0x7FFFFFFFu) | (__float_as_uint(vv) & 0x80000000u));
+                }
+                w[i] = rtn_pack2_e4m3(r[0], r[1]) | (rtn_pack2_e4m3(r[2], r[3]) << 16);   // exact; saturates beyond 448
+            }
         }
     }
     return make_uint4(w[0], w[1], w[2], w[3]);
@@ -257,11 +283,150 @@ __global__ void __launch_bounds__(kThreads) ssd_update_kernel(const UpdateParams
     }
 }
 
+// Sum four per-lane partial dots over the LPR lanes of a slot with a transposed butterfly: after
+// the first two exchanges each lane carries one of the four rows, so the remaining steps move one
+// value instead of four.  Returns the total of row j = lane_in_slot / (LPR / 4).
+template <int LPR>
+__device__ __forceinline__ float reduce4_over_slot(float d0, float d1, float d2, float d3, uint32_t lis) {
+    static_assert(LPR >= 4, "needs at least four lanes per row");
+    constexpr unsigned FULL = 0xFFFFFFFFu;
+    const bool hi1 = (lis & (LPR / 2)) != 0;
+    float k0 = hi1 ? d2 : d0, k1 = hi1 ? d3 : d1;
+    const float s0 = hi1 ? d0 : d2, s1 = hi1 ? d1 : d3;
+    k0 += __shfl_xor_sync(FULL, s0, LPR / 2);
+    k1 += __shfl_xor_sync(FULL, s1, LPR / 2);
+    const bool hi2 = (lis & (LPR / 4)) != 0;
+    float k = hi2 ? k1 : k0;
+    const float s = hi2 ? k0 : k1;
+    k += __shfl_xor_sync(FULL, s, LPR / 4);
+#pragma unroll
+    for (int off = LPR / 8; off > 0; off >>= 1) k += __shfl_xor_sync(FULL, k, off);
+    return k;
+}
+
+// The tile kernel: the same computation for the shapes that dominate (one decay per head, a head of
+// P = (kThreads / LPR) * RPS rows), one CTA per (b, h).  A head's state is one contiguous tile (16 KB for
+// 64 x 128 two-byte codes); every lane issues all RPS of its 128-bit state loads, the x row and its
+// constants before touching any of them, then walks its rows four at a time.  No guards, no idle lanes.
+template <int FMT, int RULE, int LPR, int RPS>
+__global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateParams p) {
+    constexpr int EPL = Fmt<FMT>::kEpl;
+    constexpr int N = LPR * EPL;
+    constexpr int NSLOT = kThreads / LPR;
+    constexpr unsigned FULL = 0xFFFFFFFFu;
+    static_assert(RPS % 4 == 0, "rows are processed four at a time");
+
+    const uint32_t lis = threadIdx.x % LPR;
+    const uint32_t slot = threadIdx.x / LPR;
+    const uint32_t item = blockIdx.x;
+    const uint32_t b = item / p.H;
+    const uint32_t h = item - b * p.H;
+    const uint32_t n0 = lis * EPL;
+    const uint64_t row_first = (uint64_t)item * (NSLOT * RPS) + slot * RPS;
+    const bool row_scale = (FMT == FMT_E4M3) && (p.scale_block == (uint32_t)N);
+
+    // every load of the CTA is issued here
+    uint4* sp = reinterpret_cast<uint4*>(p.state) + row_first * LPR + lis;
+    uint4 raw[RPS];
+#pragma unroll
+    for (int k = 0; k < RPS; ++k) raw[k] = sp[k * LPR];
+    float xv[RPS];
+    float sc[FMT == FMT_E4M3 ? RPS : 1];
+#pragma unroll
+    for (int k = 0; k < RPS / 4; ++k) {
+        const float4 x4 = __ldg(reinterpret_cast<const float4*>(p.x + row_first) + k);
+        xv[4 * k] = x4.x; xv[4 * k + 1] = x4.y; xv[4 * k + 2] = x4.z; xv[4 * k + 3] = x4.w;
+    }
+    if constexpr (FMT == FMT_E4M3) {
+#pragma unroll
+        for (int k = 0; k < RPS; ++k) sc[k] = row_scale ? p.scales[row_first + k] : p.scales[(row_first + k) * (N / 16) + lis];
+    }
+    float Bv[EPL], Cv[EPL];
+    {
+        const float4* Bp = reinterpret_cast<const float4*>(p.Bm + (size_t)b * N + n0);
+        const float4* Cp = reinterpret_cast<const float4*>(p.Cm + (size_t)b * N + n0);
+#pragma unroll
+        for (int i = 0; i < EPL / 4; ++i) {
+            const float4 bb = __ldg(Bp + i), cc = __ldg(Cp + i);
+            Bv[4 * i] = bb.x; Bv[4 * i + 1] = bb.y; Bv[4 * i + 2] = bb.z; Bv[4 * i + 3] = bb.w;
+            Cv[4 * i] = cc.x; Cv[4 * i + 1] = cc.y; Cv[4 * i + 2] = cc.z; Cv[4 * i + 3] = cc.w;
+        }
+    }
+    const float dtv = __ldg(p.dt + item);
+    const float a = exp_spec(__fmul_rn(dtv, __ldg(p.A + h)));
+    const float Dl = (p.D && lis == 0) ? __ldg(p.D + h) : 0.0f;     // the skip term enters the dot on one lane
+
+    LaneThreshold<FMT, RULE, LPR> thr;
+    thr.init(p.weyl, p.step_t, lis);
+    const uint32_t key0 = (uint32_t)p.sr_seed, key1 = (uint32_t)(p.sr_seed >> 32);
+    const uint64_t grow_first = row_first + (uint64_t)p.batch_base * p.H * (NSLOT * RPS);
+    uint32_t acc_row = 0;
+    uint64_t grp_row = 0;
+    if constexpr (RULE == RULE_WEYL) acc_row = thr.weyl_acc0(grow_first);
+    if constexpr (RULE == RULE_SR) grp_row = (grow_first * (uint64_t)N + n0) >> 2;
+
+#pragma unroll
+    for (int g4 = 0; g4 < RPS / 4; ++g4) {
+        float dots[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int k = g4 * 4 + u;
+            float hv[EPL];
+            unpack_lane<FMT>(raw[k], hv);
+            const float dtx = __fmul_rn(dtv, xv[k]);
+            float dot = __fmul_rn(Dl, xv[k]);
+            float amax = 0.0f;
+#pragma unroll
+            for (int j = 0; j < EPL; ++j) {
+                float hin = hv[j];
+                if constexpr (FMT == FMT_E4M3) hin = __fmul_rn(hin, sc[k]);
+                const float hn = __fmaf_rn(a, hin, __fmul_rn(dtx, Bv[j]));
+                hv[j] = hn;
+                dot = __fmaf_rn(Cv[j], hn, dot);
+                if constexpr (FMT == FMT_E4M3) amax = fmaxf(amax, fabsf(hn));
+            }
+            dots[u] = dot;
+            if constexpr (FMT == FMT_E4M3) {
+                if (row_scale) {
+#pragma unroll
+                    for (int off = LPR / 2; off > 0; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, off));
+                }
+                const float s = fmaxf(__fdiv_rn(amax, 448.0f), 1.17549435e-38f);
+                const float rinv = __fdiv_rn(1.0f, s);
+#pragma unroll
+                for (int j = 0; j < EPL; ++j) hv[j] = __fmul_rn(hv[j], rinv);
+                if (row_scale) { if (lis == 0) p.scales[row_first + k] = s; }
+                else p.scales[(row_first + k) * (N / 16) + lis] = s;
+            }
+            const uint4 packed = round_pack_lane<FMT, RULE>(hv, acc_row, p.weyl.mul_col, (uint32_t)grp_row,
+                                                             (uint32_t)(grp_row >> 32), p.step_t, p.layer, key0, key1);
+            sp[k * LPR] = packed;
+            if constexpr (RULE == RULE_WEYL) acc_row += thr.row_mul;
+            if constexpr (RULE == RULE_SR) grp_row += N / 4;
+        }
+        const float tot = reduce4_over_slot<LPR>(dots[0], dots[1], dots[2], dots[3], lis);
+        if ((lis & (LPR / 4 - 1)) == 0) p.y[row_first + g4 * 4 + lis / (LPR / 4)] = tot;
+    }
+}
+
 // Host-side launcher for one (format, rule): picks the lanes-per-row instantiation from N.
 template <int FMT, int RULE, int LPR, bool APS>
 inline cudaError_t launch_update_one(const UpdateParams& p, cudaStream_t stream) {
     UpdateParams q = p;
     const uint32_t nslot = kThreads / LPR;
+    if constexpr (!APS && LPR >= 4 && FMT != FMT_FP32) {
+        // shapes the tile kernel covers: a head of nslot * {4, 8} rows; x, y (and row scales) 16-byte aligned
+        const bool aligned = ((reinterpret_cast<uintptr_t>(q.x) | reinterpret_cast<uintptr_t>(q.y)) & 15u) == 0 &&
+                             (FMT != FMT_E4M3 || (reinterpret_cast<uintptr_t>(q.scales) & 15u) == 0);
+        if (aligned && q.P == nslot * 8u) {
+            ssd_update_tile_kernel<FMT, RULE, LPR, 8><<<q.n_items, kThreads, 0, stream>>>(q);
+            return cudaGetLastError();
+        }
+        if (aligned && q.P == nslot * 4u) {
+            ssd_update_tile_kernel<FMT, RULE, LPR, 4><<<q.n_items, kThreads, 0, stream>>>(q);
+            return cudaGetLastError();
+        }
+    }
     uint32_t spi = 1;
     while (spi < q.P && spi < nslot) spi <<= 1;        // slots per item: power of two, >= min(P, nslot)
     q.spi = spi;
