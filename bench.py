@@ -30,6 +30,11 @@ from paper_2609_39185_b200 import workloads  # noqa: E402
 
 RULE_IDS = {"rtn": 0, "sr": 1, "weyl": 2}
 NOMINAL_HBM_GBS = 8000.0
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the fused update kernel, from the ncu
+# captures summarised under profiles/ (same kernel and per-layer shape as the benchmark's launches).
+NCU_TRAFFIC_BYTES = {(5, "weyl"): 272_856_320 + 214_808_576, (5, "rtn"): 272_839_168 + 213_272_832,
+                     (3, "weyl"): 85_308_416 + 27_165_440, (3, "rtn"): 85_309_184 + 27_241_472,
+                     (4, "weyl"): 17_896_448, (4, "rtn"): 17_885_696}
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -237,7 +242,8 @@ def main():
         torch.cuda.synchronize()
 
     rule = RULE_IDS[args.rule]
-    stack = Stack(cfg, rule, batch_index_base=rank * cfg.batch)
+    from paper_2609_39185_b200.replicas import shard_batch_base
+    stack = Stack(cfg, rule, batch_index_base=shard_batch_base(rank, cfg.batch))
     xs_h, dts_h, Bs_h, Cs_h = make_ring(cfg, args.ring, 0, pin=True)
     xs, dts, Bs, Cs = (t.cuda() for t in (xs_h, dts_h, Bs_h, Cs_h))
     ys = torch.empty_like(xs)
@@ -256,10 +262,8 @@ def main():
     barrier()
     launches = ssdq.launch_count() - launches0
     clocks = sampler.stop()
-    if dist is not None:
-        tt = torch.tensor([secs], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        secs = float(tt.item())
+    from paper_2609_39185_b200.replicas import max_over_ranks
+    secs = max_over_ranks(secs, dist, "cuda")
     gbs = bytes_per_step * args.steps * world / secs / 1e9
     launch_secs = secs / (args.steps * cfg.n_layers)
     peak, peak_src = measured_peak()
@@ -271,7 +275,8 @@ def main():
             "steps_per_s": args.steps / secs, "pct_of_nominal_8tbs": 100.0 * gbs / world / NOMINAL_HBM_GBS,
             "pct_of_measured_copy": 100.0 * gbs / world / peak,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": None, "kernel": "ssd_update_kernel", "peak_source": peak_src,
+                         "traffic": None if args.batch else NCU_TRAFFIC_BYTES.get((cfg.index, args.rule)),
+                         "kernel": "ssd_update_tile_kernel" if cfg.headdim >= 32 and not cfg.a_per_state else "ssd_update_kernel", "peak_source": peak_src,
                          "algorithmic_bytes_per_launch": bytes_per_launch, "launch_us": launch_secs * 1e6},
             "clocks": clocks, "gpu_launches": int(launches)}
 
@@ -326,10 +331,7 @@ def main():
         e1.record()
         e1.synchronize()
         e2e_secs = e0.elapsed_time(e1) / 1e3
-        if dist is not None:
-            tt = torch.tensor([e2e_secs], device="cuda", dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            e2e_secs = float(tt.item())
+        e2e_secs = max_over_ranks(e2e_secs, dist, "cuda")
         line["e2e"] = {"value": bytes_per_step * e2e_steps * world / e2e_secs / 1e9, "unit": "GB/s",
                        "h2d_bytes_per_step": int(in_bytes), "d2h_bytes_per_step": int(out_bytes),
                        "ms_per_step": e2e_secs / e2e_steps * 1e3, "steps": e2e_steps,
