@@ -138,6 +138,24 @@ typedef struct {
 int ssd_decode_run(const ssdq_update_desc* layers, uint32_t n_layers, uint32_t t_first, uint32_t n_steps,
                    const ssdq_step_inputs* in, void* stream);
 
+/* Sanity metric of a quantised trajectory against its full-precision twin (Appendix B "Open-loop replay":
+ * state error = sum (h_hat - h)^2 / sum h^2): err2_per_head[h] = sum over b, p, n of (dequant(codes) - twin)^2 and
+ * ref2_per_head[h] = sum of twin^2, both DEVICE doubles [nheads], kept per head so that the caller can bin heads
+ * by memory length.  codes/scales as in ssdq_update_desc; twin [B, H, P, N] DEVICE floats.  headdim * dstate must
+ * be a multiple of 16.  `workspace` is DEVICE scratch of at least ssdq_state_error_workspace_bytes(batch, nheads)
+ * bytes, 16-byte aligned, owned by the caller; it holds per-(b, h) partial sums between the two passes (the sums
+ * over the batch are taken in a fixed order, so results are identical from run to run). */
+uint64_t ssdq_state_error_workspace_bytes(uint32_t batch, uint32_t nheads);
+int ssdq_state_error(const void* codes, const float* scales, const float* twin, uint32_t batch, uint32_t nheads,
+                     uint32_t headdim, uint32_t dstate, int format, uint32_t scale_block, double* err2_per_head,
+                     double* ref2_per_head, void* workspace, uint64_t workspace_bytes, void* stream);
+
+/* Surrogate of the paper's per-token KL (Section 4 "What we measure"; there is no vocabulary here): for each
+ * sequence b, KL(p || q) = sum_i p_i log(p_i / q_i) with p = softmax(y_ref[b, :]) and q = softmax(y_q[b, :]) over the
+ * `width` readout values of that sequence.  y_ref, y_q [batch, width] and kl_per_sequence [batch] are DEVICE floats. */
+int ssdq_readout_kl(const float* y_ref, const float* y_q, uint32_t batch, uint32_t width, float* kl_per_sequence,
+                    void* stream);
+
 /* Text of the last error on this thread ("" if none).  The pointer stays valid until the next call
  * of the library on the same thread. */
 const char* ssdq_last_error(void);

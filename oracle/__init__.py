@@ -196,3 +196,24 @@ def new_state(shape, fmt, scale_block=0):
 
 def num_threads() -> int:
     return lib().oracle_num_threads()
+
+
+# ---- sanity metrics (plain definitions, float64) ---------------------------------------------
+def state_error_per_head(codes, scales, twin, fmt, scale_block=0):
+    """Appendix B "Open-loop replay": sum (h_hat - h)^2 and sum h^2, here kept per head.
+    codes [B,H,P,N]; twin float32 [B,H,P,N].  Returns (err2 [H], ref2 [H]) float64."""
+    hq = dequantize(codes, scales, fmt, scale_block).astype(np.float64).reshape(codes.shape)
+    ref = np.asarray(twin, dtype=np.float64).reshape(codes.shape)
+    return ((hq - ref) ** 2).sum(axis=(0, 2, 3)), (ref ** 2).sum(axis=(0, 2, 3))
+
+
+def readout_kl(y_ref, y_q):
+    """KL(p || q) = sum p log(p / q) per sequence with p, q the softmax of each sequence's readout vector
+    (the per-token KL of Section 4 "What we measure", on a surrogate distribution)."""
+    a = np.asarray(y_ref, dtype=np.float64).reshape(len(y_ref), -1)
+    b = np.asarray(y_q, dtype=np.float64).reshape(len(y_q), -1)
+    lp = a - a.max(axis=1, keepdims=True)
+    lp = lp - np.log(np.exp(lp).sum(axis=1, keepdims=True))
+    lq = b - b.max(axis=1, keepdims=True)
+    lq = lq - np.log(np.exp(lq).sum(axis=1, keepdims=True))
+    return (np.exp(lp) * (lp - lq)).sum(axis=1)

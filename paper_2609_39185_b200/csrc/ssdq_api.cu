@@ -215,6 +215,34 @@ int ssd_decode_run(const ssdq_update_desc* layers, uint32_t n_layers, uint32_t t
     return SSDQ_OK;
 }
 
+uint64_t ssdq_state_error_workspace_bytes(uint32_t batch, uint32_t nheads) { return (uint64_t)batch * nheads * 16u; }
+
+int ssdq_state_error(const void* codes, const float* scales, const float* twin, uint32_t batch, uint32_t nheads,
+                     uint32_t headdim, uint32_t dstate, int format, uint32_t scale_block, double* err2_per_head,
+                     double* ref2_per_head, void* workspace, uint64_t workspace_bytes, void* stream) {
+    if (format < SSDQ_FP16 || format > SSDQ_FP32) return fail(SSDQ_ERR_UNSUPPORTED, "unknown format %d", format);
+    if (batch == 0 || nheads == 0 || headdim == 0 || dstate == 0) return fail(SSDQ_ERR_SHAPE, "sizes must be positive");
+    if (((uint64_t)headdim * dstate) % 16 != 0) return fail(SSDQ_ERR_SHAPE, "headdim * dstate must be a multiple of 16");
+    if ((uint64_t)batch * nheads > 0x7FFFFFFFull) return fail(SSDQ_ERR_SHAPE, "batch * nheads too large");
+    if (!codes || !twin || !err2_per_head || !ref2_per_head || !workspace) return fail(SSDQ_ERR_NULL, "codes, twin, outputs and workspace are required");
+    if (!aligned16(codes) || !aligned16(workspace) || !aligned4(twin)) return fail(SSDQ_ERR_ALIGN, "codes and workspace must be 16-byte aligned");
+    if (workspace_bytes < ssdq_state_error_workspace_bytes(batch, nheads)) return fail(SSDQ_ERR_SHAPE, "workspace too small");
+    if (format == SSDQ_E4M3 && (!scales || scale_block == 0 || scale_block % 16 != 0))
+        return fail(SSDQ_ERR_SHAPE, "E4M3 needs scales and a scale_block that is a multiple of 16");
+    const int rc = cuda_result(ssdq::launch_state_error(codes, scales, twin, batch, nheads, headdim * dstate, format, scale_block,
+                                                        err2_per_head, ref2_per_head, workspace, static_cast<cudaStream_t>(stream)),
+                               "state-error kernels");
+    if (rc == SSDQ_OK) g_launches.fetch_add(1, std::memory_order_relaxed);   // two kernels per call
+    return rc;
+}
+
+int ssdq_readout_kl(const float* y_ref, const float* y_q, uint32_t batch, uint32_t width, float* kl_per_sequence, void* stream) {
+    if (batch == 0 || width == 0) return fail(SSDQ_ERR_SHAPE, "batch and width must be positive");
+    if (!y_ref || !y_q || !kl_per_sequence) return fail(SSDQ_ERR_NULL, "y_ref, y_q and kl_per_sequence are required");
+    return cuda_result(ssdq::launch_readout_kl(y_ref, y_q, batch, width, kl_per_sequence, static_cast<cudaStream_t>(stream)),
+                       "readout-KL kernel");
+}
+
 const char* ssdq_last_error(void) { return g_err; }
 
 uint64_t ssdq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

@@ -57,4 +57,9 @@ cudaError_t launch_dequantize(const void* codes, const float* scales, uint64_t n
 cudaError_t launch_thresholds(int rule, const WeylConst& w, uint64_t sr_seed, uint32_t layer, uint64_t first_flat,
                               uint64_t n, uint32_t step_t, uint32_t* out, cudaStream_t s);
 
+cudaError_t launch_state_error(const void* codes, const float* scales, const float* twin, uint32_t batch, uint32_t nheads,
+                               uint32_t item_elems, int fmt, uint32_t scale_block, double* err2, double* ref2,
+                               void* workspace, cudaStream_t s);
+cudaError_t launch_readout_kl(const float* y_ref, const float* y_q, uint32_t batch, uint32_t width, float* kl, cudaStream_t s);
+
 }  // namespace ssdq

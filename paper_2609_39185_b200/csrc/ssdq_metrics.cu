@@ -1,0 +1,128 @@
+// ssdq_metrics.cu -- sanity metrics of a quantised trajectory against its full-precision twin:
+// the state error sum (h_hat - h)^2 / sum h^2 of the open-loop replay (Appendix B "Open-loop replay"),
+// kept per head so that it can be binned by memory length, and a KL divergence between softmax
+// distributions over the readout vector of each sequence (a surrogate of Section 4's per-token KL: there is
+// no vocabulary here).
+#include "ssdq_update.cuh"
+
+namespace ssdq {
+
+constexpr int kMetricThreads = 256;
+
+__device__ __forceinline__ double block_sum(double v, double* smem) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    __syncthreads();
+    if (lane == 0) smem[warp] = v;
+    __syncthreads();
+    double t = 0.0;
+    for (int w = 0; w < kMetricThreads / 32; ++w) t += smem[w];     // same order on every thread
+    return t;
+}
+
+// Pass 1: one CTA per (b, h) item; partial[item] = (sum (h_hat - h)^2, sum h^2) over the item's P*N entries.
+template <int FMT>
+__global__ void __launch_bounds__(kMetricThreads) state_error_partial_kernel(const uint4* __restrict__ codes,
+                                                                             const float* __restrict__ scales,
+                                                                             const float* __restrict__ twin,
+                                                                             uint32_t item_elems, uint32_t scale_block,
+                                                                             double2* __restrict__ partial) {
+    constexpr int EPL = Fmt<FMT>::kEpl;
+    __shared__ double smem[kMetricThreads / 32];
+    const uint64_t item = blockIdx.x;
+    const uint64_t first = item * item_elems;
+    double e2 = 0.0, r2 = 0.0;
+    for (uint32_t i = threadIdx.x * EPL; i < item_elems; i += kMetricThreads * EPL) {
+        float h[EPL];
+        unpack_lane<FMT>(codes[(first + i) / EPL], h);
+        if constexpr (FMT == FMT_E4M3) {
+            const float s = scales[(first + i) / scale_block];
+#pragma unroll
+            for (int j = 0; j < EPL; ++j) h[j] = __fmul_rn(h[j], s);
+        }
+#pragma unroll
+        for (int j = 0; j < EPL; ++j) {
+            const double ref = (double)twin[first + i + j];
+            const double d = (double)h[j] - ref;
+            e2 += d * d;
+            r2 += ref * ref;
+        }
+    }
+    e2 = block_sum(e2, smem);
+    r2 = block_sum(r2, smem);
+    if (threadIdx.x == 0) partial[item] = make_double2(e2, r2);
+}
+
+// Pass 2: one thread per head sums its items over the batch in a fixed order (run-to-run identical).
+__global__ void state_error_finish_kernel(const double2* __restrict__ partial, uint32_t batch, uint32_t nheads,
+                                          double* __restrict__ err2, double* __restrict__ ref2) {
+    const uint32_t h = blockIdx.x * blockDim.x + threadIdx.x;
+    if (h >= nheads) return;
+    double e = 0.0, r = 0.0;
+    for (uint32_t b = 0; b < batch; ++b) {
+        const double2 p = partial[(uint64_t)b * nheads + h];
+        e += p.x;
+        r += p.y;
+    }
+    err2[h] = e;
+    ref2[h] = r;
+}
+
+cudaError_t launch_state_error(const void* codes, const float* scales, const float* twin, uint32_t batch, uint32_t nheads,
+                               uint32_t item_elems, int fmt, uint32_t scale_block, double* err2, double* ref2,
+                               void* workspace, cudaStream_t s) {
+    const uint32_t n_items = batch * nheads;
+    double2* partial = reinterpret_cast<double2*>(workspace);
+    const uint4* c = reinterpret_cast<const uint4*>(codes);
+    switch (fmt) {
+        case FMT_FP16: state_error_partial_kernel<FMT_FP16><<<n_items, kMetricThreads, 0, s>>>(c, scales, twin, item_elems, scale_block, partial); break;
+        case FMT_BF16: state_error_partial_kernel<FMT_BF16><<<n_items, kMetricThreads, 0, s>>>(c, scales, twin, item_elems, scale_block, partial); break;
+        case FMT_E4M3: state_error_partial_kernel<FMT_E4M3><<<n_items, kMetricThreads, 0, s>>>(c, scales, twin, item_elems, scale_block, partial); break;
+        case FMT_FP32: state_error_partial_kernel<FMT_FP32><<<n_items, kMetricThreads, 0, s>>>(c, scales, twin, item_elems, scale_block, partial); break;
+        default: return cudaErrorInvalidValue;
+    }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    state_error_finish_kernel<<<(nheads + 127) / 128, 128, 0, s>>>(partial, batch, nheads, err2, ref2);
+    return cudaGetLastError();
+}
+
+// KL(p || q) with p = softmax(y_ref[b, :]), q = softmax(y_q[b, :]); one CTA per sequence.
+__global__ void __launch_bounds__(kMetricThreads) readout_kl_kernel(const float* __restrict__ y_ref, const float* __restrict__ y_q,
+                                                                    uint32_t width, float* __restrict__ kl) {
+    __shared__ double smem[kMetricThreads / 32];
+    __shared__ float fmax_s[2][kMetricThreads / 32];
+    const float* a = y_ref + (uint64_t)blockIdx.x * width;
+    const float* b = y_q + (uint64_t)blockIdx.x * width;
+    float ma = -INFINITY, mb = -INFINITY;
+    for (uint32_t i = threadIdx.x; i < width; i += kMetricThreads) { ma = fmaxf(ma, a[i]); mb = fmaxf(mb, b[i]); }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        ma = fmaxf(ma, __shfl_xor_sync(0xFFFFFFFFu, ma, off));
+        mb = fmaxf(mb, __shfl_xor_sync(0xFFFFFFFFu, mb, off));
+    }
+    if (threadIdx.x % 32 == 0) { fmax_s[0][threadIdx.x / 32] = ma; fmax_s[1][threadIdx.x / 32] = mb; }
+    __syncthreads();
+    for (int w = 0; w < kMetricThreads / 32; ++w) { ma = fmaxf(ma, fmax_s[0][w]); mb = fmaxf(mb, fmax_s[1][w]); }
+    // log-sum-exp of both rows, then sum p (log p - log q)
+    double sa = 0.0, sb = 0.0;
+    for (uint32_t i = threadIdx.x; i < width; i += kMetricThreads) { sa += exp((double)a[i] - ma); sb += exp((double)b[i] - mb); }
+    sa = block_sum(sa, smem);
+    sb = block_sum(sb, smem);
+    const double lza = (double)ma + log(sa), lzb = (double)mb + log(sb);
+    double acc = 0.0;
+    for (uint32_t i = threadIdx.x; i < width; i += kMetricThreads) {
+        const double lp = (double)a[i] - lza, lq = (double)b[i] - lzb;
+        acc += exp(lp) * (lp - lq);
+    }
+    acc = block_sum(acc, smem);
+    if (threadIdx.x == 0) kl[blockIdx.x] = (float)acc;
+}
+
+cudaError_t launch_readout_kl(const float* y_ref, const float* y_q, uint32_t batch, uint32_t width, float* kl, cudaStream_t s) {
+    readout_kl_kernel<<<batch, kMetricThreads, 0, s>>>(y_ref, y_q, width, kl);
+    return cudaGetLastError();
+}
+
+}  // namespace ssdq

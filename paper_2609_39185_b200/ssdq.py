@@ -17,7 +17,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libssdq.so")
 
 EXPORTS = ("weyl_offsets_init", "ssdq_thresholds_materialize", "ssd_state_update", "quantize_store",
-           "ssdq_dequantize", "ssd_decode_run", "ssdq_last_error", "ssdq_launch_count")
+           "ssdq_dequantize", "ssd_decode_run", "ssdq_state_error_workspace_bytes", "ssdq_state_error",
+           "ssdq_readout_kl", "ssdq_last_error", "ssdq_launch_count")
 
 _u32, _u64, _i32, _vp = ctypes.c_uint32, ctypes.c_uint64, ctypes.c_int32, ctypes.c_void_p
 
@@ -70,6 +71,12 @@ def lib() -> ctypes.CDLL:
         L.ssdq_dequantize.argtypes = [_vp, _vp, _u64, ctypes.c_int, _u32, _vp, _vp]
         L.ssd_decode_run.restype = ctypes.c_int
         L.ssd_decode_run.argtypes = [ctypes.POINTER(UpdateDesc), _u32, _u32, _u32, ctypes.POINTER(StepInputs), _vp]
+        L.ssdq_state_error_workspace_bytes.restype = _u64
+        L.ssdq_state_error_workspace_bytes.argtypes = [_u32, _u32]
+        L.ssdq_state_error.restype = ctypes.c_int
+        L.ssdq_state_error.argtypes = [_vp, _vp, _vp, _u32, _u32, _u32, _u32, ctypes.c_int, _u32, _vp, _vp, _vp, _u64, _vp]
+        L.ssdq_readout_kl.restype = ctypes.c_int
+        L.ssdq_readout_kl.argtypes = [_vp, _vp, _u32, _u32, _vp, _vp]
         L.ssdq_last_error.restype = ctypes.c_char_p
         L.ssdq_last_error.argtypes = []
         L.ssdq_launch_count.restype = _u64
@@ -165,6 +172,30 @@ def ssd_decode_run(layer_descs, t_first: int, n_steps: int, step_inputs: StepInp
     """n_steps decode steps over all layers on the current stream (one launch per layer per step)."""
     arr = (UpdateDesc * len(layer_descs))(*layer_descs)
     _check(lib().ssd_decode_run(arr, len(layer_descs), t_first & 0xFFFFFFFF, n_steps, ctypes.byref(step_inputs), _stream()))
+
+
+def state_error(codes, scales, twin, fmt, scale_block=0, workspace=None):
+    """Per-head sums (err2, ref2) of (dequant(codes) - twin)^2 and twin^2 as CUDA float64 tensors [H].
+    codes [B,H,P,N]; twin float32 [B,H,P,N].  `workspace` (uint8 CUDA tensor) is allocated here if not given."""
+    import torch
+    B, H, P, N = codes.shape
+    need = int(lib().ssdq_state_error_workspace_bytes(B, H))
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=codes.device)
+    err2 = torch.empty(H, dtype=torch.float64, device=codes.device)
+    ref2 = torch.empty(H, dtype=torch.float64, device=codes.device)
+    _check(lib().ssdq_state_error(_ptr(codes), _ptr(scales), _ptr(twin), B, H, P, N, fmt, scale_block, _ptr(err2), _ptr(ref2),
+                                  _ptr(workspace), workspace.numel(), _stream()))
+    return err2, ref2
+
+
+def readout_kl(y_ref, y_q):
+    """KL(softmax(y_ref[b]) || softmax(y_q[b])) per sequence; y_* float32 CUDA tensors [B, ...]."""
+    import torch
+    B = y_ref.shape[0]
+    out = torch.empty(B, dtype=torch.float32, device=y_ref.device)
+    _check(lib().ssdq_readout_kl(_ptr(y_ref), _ptr(y_q), B, y_ref[0].numel(), _ptr(out), _stream()))
+    return out
 
 
 def launch_count() -> int:
