@@ -150,6 +150,26 @@ int ssdq_state_error(const void* codes, const float* scales, const float* twin, 
                      uint32_t headdim, uint32_t dstate, int format, uint32_t scale_block, double* err2_per_head,
                      double* ref2_per_head, void* workspace, uint64_t workspace_bytes, void* stream);
 
+/* The same metric for callers that must not allocate.  (No counterpart in the paper: this entry point exists
+ * for the way the library is deployed.)  Some callers of a decode library cannot obtain device memory at the
+ * moment they want this number: a serving process that gave the whole HBM to its state/KV pool at start-up has
+ * nothing left for cudaMalloc to hand out, and a monitoring hook that runs between decode steps cannot afford
+ * cudaMalloc/cudaFree there, because both synchronise the device and would stall the decode loop.  This variant
+ * therefore takes no workspace and calls no allocating routine: its scratch (16 bytes per (b, h) pair) is a fixed
+ * array inside the library's device image, SSDQ_STATE_ERROR_STATIC_MAX_ITEMS pairs = 1 MiB, which every GPU that
+ * loads the library holds until the process exits.
+ *   - batch * nheads beyond SSDQ_STATE_ERROR_STATIC_MAX_ITEMS is rejected with SSDQ_ERR_SHAPE (use ssdq_state_error).
+ *   - The first call on each device looks up the array's address on that device (the device must be current);
+ *     make that first call before any stream capture begins.
+ *   - All calls share the one array, which keeps the contents of the last call.  Nothing in it has to start at zero
+ *     (each call overwrites every slot it later reads), but two calls that overlap on the GPU -- different streams,
+ *     or different host threads on the same device -- race on it: serialise them.
+ * Arguments and results are those of ssdq_state_error, minus the workspace. */
+#define SSDQ_STATE_ERROR_STATIC_MAX_ITEMS 65536u
+int ssdq_state_error_static(const void* codes, const float* scales, const float* twin, uint32_t batch, uint32_t nheads,
+                            uint32_t headdim, uint32_t dstate, int format, uint32_t scale_block, double* err2_per_head,
+                            double* ref2_per_head, void* stream);
+
 /* Surrogate of the paper's per-token KL (Section 4 "What we measure"; there is no vocabulary here): for each
  * sequence b, KL(p || q) = sum_i p_i log(p_i / q_i) with p = softmax(y_ref[b, :]) and q = softmax(y_q[b, :]) over the
  * `width` readout values of that sequence.  y_ref, y_q [batch, width] and kl_per_sequence [batch] are DEVICE floats. */

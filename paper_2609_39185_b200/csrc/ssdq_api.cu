@@ -98,6 +98,11 @@ cudaError_t launch_update(const ssdq::UpdateParams& p, int fmt, int rule, bool a
 
 }  // namespace
 
+namespace ssdq {
+int report_failure(int status, const char* text) { return fail(status, "%s", text); }
+void count_launches(unsigned n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+}  // namespace ssdq
+
 extern "C" {
 
 int weyl_offsets_init(ssdq_weyl* out, uint32_t layer, uint32_t seed, uint32_t block) {

@@ -60,6 +60,10 @@ cudaError_t launch_thresholds(int rule, const WeylConst& w, uint64_t sr_seed, ui
 cudaError_t launch_state_error(const void* codes, const float* scales, const float* twin, uint32_t batch, uint32_t nheads,
                                uint32_t item_elems, int fmt, uint32_t scale_block, double* err2, double* ref2,
                                void* workspace, cudaStream_t s);
+// error text / launch counter of the C ABI, for entry points defined outside ssdq_api.cu
+int report_failure(int status, const char* text);
+void count_launches(unsigned n);
+
 cudaError_t launch_readout_kl(const float* y_ref, const float* y_q, uint32_t batch, uint32_t width, float* kl, cudaStream_t s);
 
 }  // namespace ssdq

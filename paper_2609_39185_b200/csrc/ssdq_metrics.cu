@@ -3,6 +3,9 @@
 // kept per head so that it can be binned by memory length, and a KL divergence between softmax
 // distributions over the readout vector of each sequence (a surrogate of Section 4's per-token KL: there is
 // no vocabulary here).
+#include <mutex>
+
+#include "../../include/ssdq.h"
 #include "ssdq_update.cuh"
 
 namespace ssdq {
@@ -126,3 +129,62 @@ cudaError_t launch_readout_kl(const float* y_ref, const float* y_q, uint32_t bat
 }
 
 }  // namespace ssdq
+
+// ---------------------------------------------------------------------------------------------
+// ssdq_state_error_static: the state-error metric for callers that cannot hand over a workspace.
+// Its scratch (the per-(b, h) partial sums between the two passes) lives in this fixed device array,
+// which every GPU that loads the library carries until the process exits.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+constexpr uint32_t kStaticMaxItems = SSDQ_STATE_ERROR_STATIC_MAX_ITEMS;          // (b, h) pairs
+static __device__ __align__(256) double2 g_static_partials[kStaticMaxItems];    // 1 MiB
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+double2* g_static_ptr[kMaxDevices] = {};     // device address of g_static_partials, per device ordinal
+
+// In host code the name g_static_partials is only a stand-in for the symbol, not a device address: the
+// address valid on the current device has to be asked for.  Done once per device, on the first call there.
+int static_scratch_for_current_device(double2** out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return ssdq::report_failure(SSDQ_ERR_CUDA, cudaGetErrorString(e));
+    if (dev < 0 || dev >= kMaxDevices) return ssdq::report_failure(SSDQ_ERR_UNSUPPORTED, "device ordinal beyond the static table");
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+        void* ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_static_partials);
+        if (e != cudaSuccess || !ptr) return ssdq::report_failure(SSDQ_ERR_CUDA, e != cudaSuccess ? cudaGetErrorString(e) : "no address for the static scratch");
+        g_static_ptr[dev] = static_cast<double2*>(ptr);
+    }
+    *out = g_static_ptr[dev];
+    return SSDQ_OK;
+}
+
+}  // namespace
+
+extern "C" int ssdq_state_error_static(const void* codes, const float* scales, const float* twin, uint32_t batch,
+                                       uint32_t nheads, uint32_t headdim, uint32_t dstate, int format,
+                                       uint32_t scale_block, double* err2_per_head, double* ref2_per_head, void* stream) {
+    if (format < SSDQ_FP16 || format > SSDQ_FP32) return ssdq::report_failure(SSDQ_ERR_UNSUPPORTED, "unknown format");
+    if (batch == 0 || nheads == 0 || headdim == 0 || dstate == 0) return ssdq::report_failure(SSDQ_ERR_SHAPE, "sizes must be positive");
+    if (((uint64_t)headdim * dstate) % 16 != 0) return ssdq::report_failure(SSDQ_ERR_SHAPE, "headdim * dstate must be a multiple of 16");
+    if ((uint64_t)batch * nheads > kStaticMaxItems)
+        return ssdq::report_failure(SSDQ_ERR_SHAPE, "batch * nheads exceeds SSDQ_STATE_ERROR_STATIC_MAX_ITEMS (65536): "
+                                                   "use ssdq_state_error with a caller-owned workspace");
+    if (!codes || !twin || !err2_per_head || !ref2_per_head) return ssdq::report_failure(SSDQ_ERR_NULL, "codes, twin and outputs are required");
+    if ((reinterpret_cast<uintptr_t>(codes) & 15u) || (reinterpret_cast<uintptr_t>(twin) & 3u))
+        return ssdq::report_failure(SSDQ_ERR_ALIGN, "codes must be 16-byte aligned");
+    if (format == SSDQ_E4M3 && (!scales || scale_block == 0 || scale_block % 16 != 0))
+        return ssdq::report_failure(SSDQ_ERR_SHAPE, "E4M3 needs scales and a scale_block that is a multiple of 16");
+    double2* scratch = nullptr;
+    const int rc = static_scratch_for_current_device(&scratch);
+    if (rc != SSDQ_OK) return rc;
+    // every partial the second pass reads is written by the first pass of this same call: nothing has to be cleared
+    const cudaError_t e = ssdq::launch_state_error(codes, scales, twin, batch, nheads, headdim * dstate, format, scale_block,
+                                                   err2_per_head, ref2_per_head, scratch, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return ssdq::report_failure(SSDQ_ERR_CUDA, cudaGetErrorString(e));
+    ssdq::count_launches(2);
+    return SSDQ_OK;
+}

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libssdq.so")
 
 EXPORTS = ("weyl_offsets_init", "ssdq_thresholds_materialize", "ssd_state_update", "quantize_store",
            "ssdq_dequantize", "ssd_decode_run", "ssdq_state_error_workspace_bytes", "ssdq_state_error",
-           "ssdq_readout_kl", "ssdq_last_error", "ssdq_launch_count")
+           "ssdq_state_error_static", "ssdq_readout_kl", "ssdq_last_error", "ssdq_launch_count")
 
 _u32, _u64, _i32, _vp = ctypes.c_uint32, ctypes.c_uint64, ctypes.c_int32, ctypes.c_void_p
 
@@ -75,6 +75,8 @@ def lib() -> ctypes.CDLL:
         L.ssdq_state_error_workspace_bytes.argtypes = [_u32, _u32]
         L.ssdq_state_error.restype = ctypes.c_int
         L.ssdq_state_error.argtypes = [_vp, _vp, _vp, _u32, _u32, _u32, _u32, ctypes.c_int, _u32, _vp, _vp, _vp, _u64, _vp]
+        L.ssdq_state_error_static.restype = ctypes.c_int
+        L.ssdq_state_error_static.argtypes = [_vp, _vp, _vp, _u32, _u32, _u32, _u32, ctypes.c_int, _u32, _vp, _vp, _vp]
         L.ssdq_readout_kl.restype = ctypes.c_int
         L.ssdq_readout_kl.argtypes = [_vp, _vp, _u32, _u32, _vp, _vp]
         L.ssdq_last_error.restype = ctypes.c_char_p
@@ -187,6 +189,20 @@ def state_error(codes, scales, twin, fmt, scale_block=0, workspace=None):
     _check(lib().ssdq_state_error(_ptr(codes), _ptr(scales), _ptr(twin), B, H, P, N, fmt, scale_block, _ptr(err2), _ptr(ref2),
                                   _ptr(workspace), workspace.numel(), _stream()))
     return err2, ref2
+
+
+STATE_ERROR_STATIC_MAX_ITEMS = 65536
+
+
+def state_error_static(codes, scales, twin, fmt, err2, ref2, scale_block=0):
+    """ssdq_state_error_static: the per-head state-error sums written into the caller's float64 CUDA tensors
+    `err2`, `ref2` [H] without any device allocation -- the scratch is a fixed 1 MiB array inside the library, so
+    batch * nheads may not exceed STATE_ERROR_STATIC_MAX_ITEMS, calls on one device must not overlap, and the
+    first call on a device should come before any stream capture.  For callers (a serving process whose pool
+    owns all of HBM, a hook inside the decode loop) that cannot call cudaMalloc."""
+    B, H, P, N = codes.shape
+    _check(lib().ssdq_state_error_static(_ptr(codes), _ptr(scales), _ptr(twin), B, H, P, N, fmt, scale_block,
+                                         _ptr(err2), _ptr(ref2), _stream()))
 
 
 def readout_kl(y_ref, y_q):
