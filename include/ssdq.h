@@ -138,6 +138,18 @@ typedef struct {
 int ssd_decode_run(const ssdq_update_desc* layers, uint32_t n_layers, uint32_t t_first, uint32_t n_steps,
                    const ssdq_step_inputs* in, void* stream);
 
+/* The same driver for callers whose per-step inputs and outputs live in HOST memory (the usual case when the
+ * rest of the model runs elsewhere): `host` describes HOST arrays (page-locked memory for full speed) laid out like
+ * ssdq_step_inputs, the inputs of step t at ring slot (t - t_first) % host->ring and its y written to the same
+ * slot; `staging` describes caller-owned DEVICE buffers with 2 to 8 ring slots and the same strides as `host`.
+ * Per step: the inputs of all layers go host -> staging on an internal copy stream, the fused updates run on
+ * `stream`, y goes staging -> host on a second internal copy stream; events chain the three so that copy-in of step
+ * t+1, compute of step t and copy-out of step t-1 overlap.  When all work enqueued on `stream` has completed,
+ * every y has reached the host.  The state never leaves the device.  The two streams and the events are created
+ * on the first call on a device (host-side driver resources, no device memory).  One call at a time per device. */
+int ssd_decode_run_host(const ssdq_update_desc* layers, uint32_t n_layers, uint32_t t_first, uint32_t n_steps,
+                        const ssdq_step_inputs* host, const ssdq_step_inputs* staging, void* stream);
+
 /* Sanity metric of a quantised trajectory against its full-precision twin (Appendix B "Open-loop replay":
  * state error = sum (h_hat - h)^2 / sum h^2): err2_per_head[h] = sum over b, p, n of (dequant(codes) - twin)^2 and
  * ref2_per_head[h] = sum of twin^2, both DEVICE doubles [nheads], kept per head so that the caller can bin heads

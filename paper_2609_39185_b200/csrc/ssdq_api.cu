@@ -5,6 +5,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 
 #include "../../include/ssdq.h"
 #include "ssdq_internal.h"
@@ -94,6 +95,46 @@ cudaError_t launch_update(const ssdq::UpdateParams& p, int fmt, int rule, bool a
         case SSDQ_FP32: return ssdq::launch_update_fp32(p, rule, aps, s);
         default: return cudaErrorInvalidValue;
     }
+}
+
+}  // namespace
+
+namespace {
+
+// Host-side resources of the host-buffer driver, one set per device: two copy streams and the events that
+// chain copy-in -> compute -> copy-out per staging slot.  Created on first use; no device memory.
+constexpr uint32_t kMaxStagingSlots = 8;
+struct HostPipe {
+    std::mutex mutex;
+    bool ready = false;
+    cudaStream_t h2d = nullptr, d2h = nullptr;
+    cudaEvent_t start = nullptr;
+    cudaEvent_t loaded[kMaxStagingSlots] = {}, computed[kMaxStagingSlots] = {}, stored[kMaxStagingSlots] = {};
+};
+HostPipe g_pipes[64];
+std::mutex g_pipes_mutex;
+
+int host_pipe_for_current_device(HostPipe** out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return fail(SSDQ_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+    if (dev < 0 || dev >= 64) return fail(SSDQ_ERR_UNSUPPORTED, "device ordinal %d beyond the table", dev);
+    std::lock_guard<std::mutex> lock(g_pipes_mutex);
+    HostPipe& hp = g_pipes[dev];
+    if (!hp.ready) {
+        if ((e = cudaStreamCreateWithFlags(&hp.h2d, cudaStreamNonBlocking)) != cudaSuccess ||
+            (e = cudaStreamCreateWithFlags(&hp.d2h, cudaStreamNonBlocking)) != cudaSuccess ||
+            (e = cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming)) != cudaSuccess)
+            return fail(SSDQ_ERR_CUDA, "stream/event creation: %s", cudaGetErrorString(e));
+        for (uint32_t i = 0; i < kMaxStagingSlots; ++i)
+            if ((e = cudaEventCreateWithFlags(&hp.loaded[i], cudaEventDisableTiming)) != cudaSuccess ||
+                (e = cudaEventCreateWithFlags(&hp.computed[i], cudaEventDisableTiming)) != cudaSuccess ||
+                (e = cudaEventCreateWithFlags(&hp.stored[i], cudaEventDisableTiming)) != cudaSuccess)
+                return fail(SSDQ_ERR_CUDA, "event creation: %s", cudaGetErrorString(e));
+        hp.ready = true;
+    }
+    *out = &hp;
+    return SSDQ_OK;
 }
 
 }  // namespace
@@ -246,6 +287,82 @@ int ssdq_readout_kl(const float* y_ref, const float* y_q, uint32_t batch, uint32
     if (!y_ref || !y_q || !kl_per_sequence) return fail(SSDQ_ERR_NULL, "y_ref, y_q and kl_per_sequence are required");
     return cuda_result(ssdq::launch_readout_kl(y_ref, y_q, batch, width, kl_per_sequence, static_cast<cudaStream_t>(stream)),
                        "readout-KL kernel");
+}
+
+int ssd_decode_run_host(const ssdq_update_desc* layers, uint32_t n_layers, uint32_t t_first, uint32_t n_steps,
+                        const ssdq_step_inputs* host, const ssdq_step_inputs* staging, void* stream) {
+    if (!layers || !host || !staging) return fail(SSDQ_ERR_NULL, "layers, host and staging are required");
+    if (n_layers == 0 || host->ring == 0) return fail(SSDQ_ERR_SHAPE, "n_layers and host ring must be positive");
+    if (staging->ring < 2 || staging->ring > kMaxStagingSlots) return fail(SSDQ_ERR_SHAPE, "staging ring must hold 2 to 8 slots");
+    if (host->stride_x != staging->stride_x || host->stride_dt != staging->stride_dt || host->stride_B != staging->stride_B ||
+        host->stride_C != staging->stride_C || host->stride_y != staging->stride_y)
+        return fail(SSDQ_ERR_SHAPE, "host and staging strides must be equal");
+    if (!host->x || !host->dt || !host->Bm || !host->Cm || !host->y) return fail(SSDQ_ERR_NULL, "host x, dt, Bm, Cm and y are required");
+    for (uint32_t l = 0; l < n_layers; ++l) {
+        const int rc = check_layer(&layers[l]);
+        if (rc != SSDQ_OK) return rc;
+    }
+    for (uint32_t sl = 0; sl < staging->ring; ++sl)
+        for (uint32_t l = 0; l < n_layers; ++l) {
+            const uint64_t k = (uint64_t)sl * n_layers + l;
+            const int rc = check_step_ptrs(staging->x + k * staging->stride_x, staging->dt + k * staging->stride_dt,
+                                           staging->Bm + k * staging->stride_B, staging->Cm + k * staging->stride_C,
+                                           staging->y + k * staging->stride_y);
+            if (rc != SSDQ_OK) return rc;
+        }
+    if (n_steps == 0) return SSDQ_OK;
+    cudaStream_t compute = static_cast<cudaStream_t>(stream);
+    HostPipe* hp = nullptr;
+    int rc = host_pipe_for_current_device(&hp);
+    if (rc != SSDQ_OK) return rc;
+    std::lock_guard<std::mutex> lock(hp->mutex);
+#define SSDQ_TRY(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return fail(SSDQ_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_)); } while (0)
+    // staging slots may still be read by earlier work on the caller's stream
+    SSDQ_TRY(cudaEventRecord(hp->start, compute));
+    SSDQ_TRY(cudaStreamWaitEvent(hp->h2d, hp->start, 0));
+    const uint32_t S = staging->ring;
+    const uint64_t L = n_layers;
+    for (uint32_t i = 0; i < n_steps; ++i) {
+        const uint32_t sl = i % S;
+        const uint64_t hk = (uint64_t)(i % host->ring) * L, dk = (uint64_t)sl * L;
+        // inputs of step i: host slot -> staging slot, once the launches that last used the slot are done
+        if (i >= S) SSDQ_TRY(cudaStreamWaitEvent(hp->h2d, hp->computed[sl], 0));
+        SSDQ_TRY(cudaMemcpyAsync(const_cast<float*>(staging->x) + dk * staging->stride_x, host->x + hk * host->stride_x,
+                                 L * host->stride_x * sizeof(float), cudaMemcpyHostToDevice, hp->h2d));
+        SSDQ_TRY(cudaMemcpyAsync(const_cast<float*>(staging->dt) + dk * staging->stride_dt, host->dt + hk * host->stride_dt,
+                                 L * host->stride_dt * sizeof(float), cudaMemcpyHostToDevice, hp->h2d));
+        SSDQ_TRY(cudaMemcpyAsync(const_cast<float*>(staging->Bm) + dk * staging->stride_B, host->Bm + hk * host->stride_B,
+                                 L * host->stride_B * sizeof(float), cudaMemcpyHostToDevice, hp->h2d));
+        SSDQ_TRY(cudaMemcpyAsync(const_cast<float*>(staging->Cm) + dk * staging->stride_C, host->Cm + hk * host->stride_C,
+                                 L * host->stride_C * sizeof(float), cudaMemcpyHostToDevice, hp->h2d));
+        SSDQ_TRY(cudaEventRecord(hp->loaded[sl], hp->h2d));
+        // the fused updates of step i, once its inputs have landed and the slot's previous y has left
+        SSDQ_TRY(cudaStreamWaitEvent(compute, hp->loaded[sl], 0));
+        if (i >= S) SSDQ_TRY(cudaStreamWaitEvent(compute, hp->stored[sl], 0));
+        for (uint32_t l = 0; l < n_layers; ++l) {
+            const uint64_t k = dk + l;
+            ssdq::UpdateParams p = make_params(&layers[l], t_first + i);
+            p.x = staging->x + k * staging->stride_x;
+            p.dt = staging->dt + k * staging->stride_dt;
+            p.Bm = staging->Bm + k * staging->stride_B;
+            p.Cm = staging->Cm + k * staging->stride_C;
+            p.y = staging->y + k * staging->stride_y;
+            rc = cuda_result(launch_update(p, layers[l].format, layers[l].rule, layers[l].a_per_state != 0, compute),
+                             "state-update kernel");
+            if (rc != SSDQ_OK) return rc;
+        }
+        SSDQ_TRY(cudaEventRecord(hp->computed[sl], compute));
+        // y of step i back to the host
+        SSDQ_TRY(cudaStreamWaitEvent(hp->d2h, hp->computed[sl], 0));
+        SSDQ_TRY(cudaMemcpyAsync(host->y + hk * host->stride_y, staging->y + dk * staging->stride_y,
+                                 L * host->stride_y * sizeof(float), cudaMemcpyDeviceToHost, hp->d2h));
+        SSDQ_TRY(cudaEventRecord(hp->stored[sl], hp->d2h));
+    }
+    // the caller's stream is complete only when every y has reached the host
+    const uint32_t used = n_steps < S ? n_steps : S;
+    for (uint32_t sl = 0; sl < used; ++sl) SSDQ_TRY(cudaStreamWaitEvent(compute, hp->stored[sl], 0));
+#undef SSDQ_TRY
+    return SSDQ_OK;
 }
 
 const char* ssdq_last_error(void) { return g_err; }

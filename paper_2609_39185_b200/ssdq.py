@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libssdq.so")
 
 EXPORTS = ("weyl_offsets_init", "ssdq_thresholds_materialize", "ssd_state_update", "quantize_store",
-           "ssdq_dequantize", "ssd_decode_run", "ssdq_state_error_workspace_bytes", "ssdq_state_error",
+           "ssdq_dequantize", "ssd_decode_run", "ssd_decode_run_host", "ssdq_state_error_workspace_bytes", "ssdq_state_error",
            "ssdq_state_error_static", "ssdq_readout_kl", "ssdq_last_error", "ssdq_launch_count")
 
 _u32, _u64, _i32, _vp = ctypes.c_uint32, ctypes.c_uint64, ctypes.c_int32, ctypes.c_void_p
@@ -71,6 +71,9 @@ def lib() -> ctypes.CDLL:
         L.ssdq_dequantize.argtypes = [_vp, _vp, _u64, ctypes.c_int, _u32, _vp, _vp]
         L.ssd_decode_run.restype = ctypes.c_int
         L.ssd_decode_run.argtypes = [ctypes.POINTER(UpdateDesc), _u32, _u32, _u32, ctypes.POINTER(StepInputs), _vp]
+        L.ssd_decode_run_host.restype = ctypes.c_int
+        L.ssd_decode_run_host.argtypes = [ctypes.POINTER(UpdateDesc), _u32, _u32, _u32, ctypes.POINTER(StepInputs),
+                                          ctypes.POINTER(StepInputs), _vp]
         L.ssdq_state_error_workspace_bytes.restype = _u64
         L.ssdq_state_error_workspace_bytes.argtypes = [_u32, _u32]
         L.ssdq_state_error.restype = ctypes.c_int
@@ -212,6 +215,15 @@ def readout_kl(y_ref, y_q):
     out = torch.empty(B, dtype=torch.float32, device=y_ref.device)
     _check(lib().ssdq_readout_kl(_ptr(y_ref), _ptr(y_q), B, y_ref[0].numel(), _ptr(out), _stream()))
     return out
+
+
+def ssd_decode_run_host(layer_descs, t_first: int, n_steps: int, host_io: StepInputs, staging: StepInputs):
+    """n_steps decode steps with per-step inputs in (pinned) HOST tensors and y returned to HOST tensors, copies
+    overlapped with compute.  `host_io` and `staging` come from make_step_inputs on host and device tensors of
+    identical per-slot shapes; staging needs 2 to 8 ring slots.  Synchronise the current stream before reading y."""
+    arr = (UpdateDesc * len(layer_descs))(*layer_descs)
+    _check(lib().ssd_decode_run_host(arr, len(layer_descs), t_first & 0xFFFFFFFF, n_steps, ctypes.byref(host_io),
+                                     ctypes.byref(staging), _stream()))
 
 
 def launch_count() -> int:

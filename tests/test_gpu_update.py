@@ -209,3 +209,38 @@ def test_ring_reuses_inputs():
         oracle.state_update(st, None, cfg.fmt, 0, x, dt, A, Bm, Cm, D, oracle.WEYL, 1 + i, weyl_block=16)
     torch.cuda.synchronize()
     assert np.array_equal(codes_to_host(state, cfg.fmt), st)
+
+
+@pytest.mark.parametrize("staging_slots,host_ring", [(2, 12), (3, 12), (2, 4)])
+def test_host_buffer_driver_equals_device_driver(staging_slots, host_ring):
+    """ssd_decode_run_host (pinned host inputs, y back to host, copies overlapped with compute) produces the
+    bits of ssd_decode_run on device-resident inputs."""
+    cfg = workloads.CONFIGS[1].with_batch(3)
+    L, T = 2, 12
+    params = [workloads.layer_params(cfg, l, l) for l in range(L)]
+    ins = [[workloads.step_inputs(cfg, 1 + (t % host_ring), l, l) for l in range(L)] for t in range(T)]
+    stack_h = lambda i: torch.from_numpy(np.stack([np.stack([ins[t][l][i] for l in range(L)]) for t in range(host_ring)])).pin_memory()
+    xs_h, dts_h, Bs_h, Cs_h = (stack_h(i) for i in range(4))
+    ys_h = torch.zeros_like(xs_h).pin_memory()
+
+    def fresh():
+        states = [torch.zeros(cfg.state_shape, dtype=torch.int16, device="cuda") for _ in range(L)]
+        descs = [ssdq.make_desc(states[l], None, cfg.fmt, A=to_dev(params[l][0]), D=to_dev(params[l][1]), rule=ssdq.WEYL,
+                                weyl=ssdq.weyl_offsets_init(l, 0, cfg.weyl_block), layer=l) for l in range(L)]
+        return states, descs
+
+    s1, d1 = fresh()
+    xs, dts, Bs, Cs = (t.cuda() for t in (xs_h, dts_h, Bs_h, Cs_h))
+    ys = torch.zeros_like(xs)
+    ssdq.ssd_decode_run(d1, 1, T, ssdq.make_step_inputs(xs, dts, Bs, Cs, ys))
+    s2, d2 = fresh()
+    stg = [torch.zeros((staging_slots,) + tuple(t.shape[1:]), dtype=torch.float32, device="cuda") for t in (xs_h, dts_h, Bs_h, Cs_h, ys_h)]
+    for _ in range(2):          # twice: the second call reuses the driver's streams and events
+        for st in s2:
+            st.zero_()
+        ys_h.zero_()
+        ssdq.ssd_decode_run_host(d2, 1, T, ssdq.make_step_inputs(xs_h, dts_h, Bs_h, Cs_h, ys_h), ssdq.make_step_inputs(*stg))
+        torch.cuda.current_stream().synchronize()
+        for l in range(L):
+            assert torch.equal(s1[l], s2[l])
+        assert torch.equal(ys.cpu(), ys_h)
