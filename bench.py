@@ -199,6 +199,32 @@ def workload_config(cfg, args):
             "parallelism": f"replicas x{args.gpus} (batch shards, no collective)"}
 
 
+def sweep_batch(args, cfg):
+    """Decode steps/s and algorithmic GB/s of the whole stack for each batch size and rule (one JSON line)."""
+    import torch
+    from paper_2609_39185_b200 import ssdq
+    rows = []
+    for b in [int(v) for v in args.sweep_batch.split(",")]:
+        c = cfg.with_batch(b)
+        stack = Stack(c, RULE_IDS["rtn"])
+        xs, dts, Bs, Cs = (t.cuda() for t in make_ring(c, args.ring, 0))
+        sin = ssdq.make_step_inputs(xs, dts, Bs, Cs, torch.empty_like(xs))
+        row = {"batch": b, "state_bytes": c.state_bytes_per_layer() * c.n_layers}
+        stack.run(1, args.warmup, sin)
+        torch.cuda.synchronize()
+        for _ in range(3):      # interleaved rounds, best of three per rule
+            for name, rid in RULE_IDS.items():
+                stack.set_rule(rid)
+                secs = time_steps(stack, sin, 1, args.steps)
+                sps = args.steps / secs
+                if sps > row.get(name, {}).get("steps_per_s", 0.0):
+                    row[name] = {"steps_per_s": sps, "gbs": c.algorithmic_bytes_per_layer_step() * c.n_layers * sps / 1e9}
+        rows.append(row)
+        del stack, xs, dts, Bs, Cs, sin
+        torch.cuda.empty_cache()
+    print(json.dumps({"metric": "decode_steps_per_s_vs_batch", "config": cfg.name, "layers": cfg.n_layers, "rows": rows}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -210,6 +236,7 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override the configuration's batch")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling captures)")
     ap.add_argument("--ring", type=int, default=4, help="distinct decode steps of inputs kept resident")
+    ap.add_argument("--sweep-batch", default="", help="comma-separated batch sizes: print steps/s per rule for each, then exit")
     ap.add_argument("--no-extras", action="store_true", help="skip the per-rule sweep, e2e and CPU baseline")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
@@ -241,6 +268,8 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    if args.sweep_batch:
+        return sweep_batch(args, cfg)
     rule = RULE_IDS[args.rule]
     from paper_2609_39185_b200.replicas import shard_batch_base
     stack = Stack(cfg, rule, batch_index_base=shard_batch_base(rank, cfg.batch))

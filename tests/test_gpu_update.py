@@ -41,8 +41,17 @@ def test_config4_e4m3_full_size_few_steps(rule):
 
 
 @pytest.mark.parametrize("rule", RULES)
-def test_config4_long_horizon_on_one_sequence(rule):
-    run_parity(CFG[4], rule, 768, batch_slice=slice(31, 32), batch_index_base=31, check_every=64)
+def test_config4_full_horizon_on_one_sequence(rule):
+    # all 4096 quantised steps (the slow heads' increments stay below half an E4M3 step throughout)
+    run_parity(CFG[4], rule, CFG[4].steps, batch_slice=slice(31, 32), batch_index_base=31, check_every=256)
+
+
+@pytest.mark.parametrize("rule", RULES)
+def test_config5_full_horizon_on_the_last_two_sequences(rule):
+    # layer 7 with its own seed, all 1024 steps, sequences 126 and 127 addressed by their global index
+    cfg = CFG[5]
+    run_parity(cfg, rule, cfg.steps, layer=7, seed=workloads.layer_seed(cfg, 0, 7), batch_slice=slice(126, 128),
+               batch_index_base=126, sr_seed=7, check_every=128)
 
 
 @pytest.mark.parametrize("rule", RULES)
