@@ -15,10 +15,17 @@ import subprocess
 import numpy as np
 
 FP16, BF16, E4M3, FP32 = 0, 1, 2, 3
+INT8, INT7, INT6, INT4 = 4, 5, 6, 7          # symmetric block-absmax integers, one int8 per entry
+INT_QMAX = {INT8: 127, INT7: 63, INT6: 31, INT4: 7}
 RTN, SR, WEYL = 0, 1, 2
-FORMAT_NAMES = {FP16: "fp16", BF16: "bf16", E4M3: "e4m3", FP32: "fp32"}
+FORMAT_NAMES = {FP16: "fp16", BF16: "bf16", E4M3: "e4m3", FP32: "fp32", INT8: "int8", INT7: "int7", INT6: "int6", INT4: "int4"}
 RULE_NAMES = {RTN: "rtn", SR: "sr", WEYL: "weyl"}
-CODE_DTYPE = {FP16: np.uint16, BF16: np.uint16, E4M3: np.uint8, FP32: np.uint32}
+CODE_DTYPE = {FP16: np.uint16, BF16: np.uint16, E4M3: np.uint8, FP32: np.uint32, INT8: np.uint8, INT7: np.uint8,
+              INT6: np.uint8, INT4: np.uint8}
+
+
+def has_block_scale(fmt):
+    return fmt == E4M3 or fmt in INT_QMAX
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "ssdq_oracle.cpp")
@@ -168,7 +175,7 @@ def quantize_store(src, fmt, rule, step_t, *, scale_block=0, layer=0, weyl_seed=
     src = _f32(src)
     n_rows, row_len = src.shape
     codes = np.zeros((n_rows, row_len), dtype=CODE_DTYPE[fmt])
-    scales = np.zeros((n_rows, row_len // scale_block), dtype=np.float32) if fmt == E4M3 else None
+    scales = np.zeros((n_rows, row_len // scale_block), dtype=np.float32) if has_block_scale(fmt) else None
     rc = lib().oracle_quantize_store(_ptr(src), _ptr(codes), _ptr(scales), n_rows, row_len, fmt, scale_block, rule,
                                      layer, weyl_seed, weyl_block, sr_seed, row_index_base, step_t)
     if rc != 0:
@@ -188,7 +195,7 @@ def new_state(shape, fmt, scale_block=0):
     Bsz, H, P, N = shape
     state = np.zeros(shape, dtype=CODE_DTYPE[fmt])
     scales = None
-    if fmt == E4M3:
+    if has_block_scale(fmt):
         n_scales = Bsz * H if scale_block == P * N and scale_block != N else Bsz * H * P * (N // scale_block)
         scales = np.full(n_scales, np.finfo(np.float32).tiny, dtype=np.float32)
     return state, scales

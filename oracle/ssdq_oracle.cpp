@@ -19,6 +19,7 @@
 //   * RTN / SR / Weyl thresholds                                -- Section 2 "Rounding with a threshold"
 //   * 32-bit Weyl accumulator, top 24 bits, R2 offsets          -- Appendix B "Dithers"
 //   * FP16 / BF16 / FP8-E4M3 + FP32 block scale max|h| / 448    -- Appendix B "Formats"
+//   * INT8/7/6/4 symmetric block-absmax, FP32 scale, clamp     -- Appendix B "Formats" (INTb)
 //
 // Pins (tests/test_oracle_*.py): Weyl 0.618, 0.236, 0.854; Philox known answers; RTN equal to
 // library casts; dithered rounding equal to exact rational arithmetic; Proposition 1 identity,
@@ -39,7 +40,8 @@
 
 namespace {
 
-enum Format { FMT_FP16 = 0, FMT_BF16 = 1, FMT_E4M3 = 2, FMT_FP32 = 3 /* no rounding: the fp32-state twin */ };
+enum Format { FMT_FP16 = 0, FMT_BF16 = 1, FMT_E4M3 = 2, FMT_FP32 = 3 /* no rounding: the fp32-state twin */,
+              FMT_INT8 = 4, FMT_INT7 = 5, FMT_INT6 = 6, FMT_INT4 = 7 /* symmetric block-absmax integers in an int8 container */ };
 enum Rule { RULE_RTN = 0, RULE_SR = 1, RULE_WEYL = 2 };
 
 struct FormatSpec {
@@ -60,6 +62,14 @@ FormatSpec spec_of(int fmt) {
         default:       return {23, -126, 127, 8, (double)FLT_MAX};
     }
 }
+
+// Appendix B "Formats", INTb: symmetric, q_max = 2^(b-1) - 1, block scale s = max|h| / q_max kept in FP32,
+// values clamped to [-q_max, q_max].  The grid is uniform (step 1 in units of s), so Eq. 2 is floor(v + u).
+bool is_int_format(int fmt) { return fmt >= FMT_INT8 && fmt <= FMT_INT4; }
+int int_qmax(int fmt) {
+    switch (fmt) { case FMT_INT8: return 127; case FMT_INT7: return 63; case FMT_INT6: return 31; default: return 7; }
+}
+bool has_block_scale(int fmt) { return fmt == FMT_E4M3 || is_int_format(fmt); }
 
 // ------------------------------------------------------------------------------------------
 // Thresholds.  U is a 24-bit integer, u = U / 2^24 (Appendix B "Dithers": "the top 24 bits
@@ -133,6 +143,15 @@ uint32_t threshold_u24(const RuleParams& rp, uint64_t flat, uint32_t t) {
 // ------------------------------------------------------------------------------------------
 float round_on_grid(float v, int fmt, int rule, uint32_t U) {
     if (fmt == FMT_FP32) return v;
+    if (is_int_format(fmt)) {
+        if (std::isnan(v)) return v;
+        const double q = (double)int_qmax(fmt);
+        if (std::isinf(v)) return (float)std::copysign(q, (double)v);
+        // v has at most 24 significant bits and u is a multiple of 2^-24: the sum is exact in double
+        double K = (rule == RULE_RTN) ? std::nearbyint((double)v) : std::floor((double)v + std::ldexp((double)U, -24));
+        K = std::min(std::max(K, -q), q);
+        return (float)(K == 0.0 ? 0.0 : K);   // an integer zero has no sign
+    }
     const FormatSpec fs = spec_of(fmt);
     if (std::isnan(v)) return v;
     if (std::isinf(v)) return std::copysign((float)fs.max_finite, v);
@@ -159,6 +178,7 @@ float round_on_grid(float v, int fmt, int rule, uint32_t U) {
 uint32_t encode(float q, int fmt) {
     const FormatSpec fs = spec_of(fmt);
     if (fmt == FMT_FP32) { uint32_t b; std::memcpy(&b, &q, 4); return b; }
+    if (is_int_format(fmt)) return (uint32_t)(uint8_t)(int8_t)(int)q;   // two's complement byte
     const uint32_t sign = std::signbit(q) ? 1u : 0u;
     const int total_bits = 1 + fs.exp_bits + fs.mant_bits;
     uint32_t field_e = 0, field_m = 0;
@@ -182,6 +202,7 @@ uint32_t encode(float q, int fmt) {
 
 float decode(uint32_t code, int fmt) {
     if (fmt == FMT_FP32) { float f; std::memcpy(&f, &code, 4); return f; }
+    if (is_int_format(fmt)) return (float)(int8_t)(uint8_t)code;
     const FormatSpec fs = spec_of(fmt);
     const int total_bits = 1 + fs.exp_bits + fs.mant_bits;
     const uint32_t sign = (code >> (total_bits - 1)) & 1u;
@@ -201,7 +222,7 @@ float decode(uint32_t code, int fmt) {
     return (float)(sign ? -a : a);
 }
 
-int code_bytes(int fmt) { return fmt == FMT_E4M3 ? 1 : (fmt == FMT_FP32 ? 4 : 2); }
+int code_bytes(int fmt) { return (fmt == FMT_E4M3 || is_int_format(fmt)) ? 1 : (fmt == FMT_FP32 ? 4 : 2); }
 
 uint32_t load_code(const void* base, uint64_t i, int fmt) {
     switch (code_bytes(fmt)) {
@@ -248,7 +269,10 @@ float exp_spec(float z) {
 // Block scale of the E4M3 store: s = max|h'| / 448 in FP32 (Appendix B "Formats"), floored at the
 // smallest normal number so that an all-zero block is well defined.  Entries are multiplied by
 // 1/s, rounded once per block, instead of being divided by s one by one.
-float block_scale(float amax) { return std::max(amax / 448.0f, FLT_MIN); }
+float block_scale(float amax, int fmt) {
+    const float top = is_int_format(fmt) ? (float)int_qmax(fmt) : 448.0f;
+    return std::max(amax / top, FLT_MIN);
+}
 
 }  // namespace
 
@@ -286,13 +310,13 @@ int oracle_state_update(void* state, float* scales, int fmt, uint32_t scale_bloc
                         const float* Bm, const float* Cm, const float* D, float* y,
                         int rule, uint32_t layer, uint32_t weyl_seed, uint32_t weyl_block, uint64_t sr_seed,
                         uint32_t batch_index_base, uint32_t step_t) {
-    if (fmt == FMT_E4M3) {
+    if (has_block_scale(fmt)) {
         if (scale_block == 0 || !scales) return -1;
         if (!(scale_block == P * N || N % scale_block == 0)) return -1;
     }
     if (rule == RULE_WEYL && (weyl_block == 0 || N % weyl_block != 0)) return -1;
     const RuleParams rp{rule, layer, weyl_seed, weyl_block, sr_seed};
-    const bool head_scale = (fmt == FMT_E4M3 && scale_block == P * N && scale_block != N);
+    const bool head_scale = (has_block_scale(fmt) && scale_block == P * N && scale_block != N);
     const int64_t BH = (int64_t)B * H;
 #pragma omp parallel for schedule(static)
     for (int64_t bh = 0; bh < BH; ++bh) {
@@ -306,7 +330,7 @@ int oracle_state_update(void* state, float* scales, int fmt, uint32_t scale_bloc
             for (uint32_t n = 0; n < N; ++n) {
                 const uint64_t local = ((uint64_t)bh * P + p) * N + n;
                 float hv = decode(load_code(state, local, fmt), fmt);
-                if (fmt == FMT_E4M3) {
+                if (has_block_scale(fmt)) {
                     const uint64_t sidx = head_scale ? (uint64_t)bh : local / scale_block;
                     hv = hv * scales[sidx];
                 }
@@ -323,20 +347,20 @@ int oracle_state_update(void* state, float* scales, int fmt, uint32_t scale_bloc
         }
         // write-back: block scale (E4M3), threshold, Eq. 2, encode
         const uint64_t head_elems = (uint64_t)P * N;
-        const uint64_t blk = (fmt == FMT_E4M3) ? scale_block : head_elems;
+        const uint64_t blk = has_block_scale(fmt) ? scale_block : head_elems;
         for (uint64_t s0 = 0; s0 < head_elems; s0 += blk) {
             float rinv = 1.0f;
-            if (fmt == FMT_E4M3) {
+            if (has_block_scale(fmt)) {
                 float amax = 0.0f;
                 for (uint64_t i = s0; i < s0 + blk; ++i) amax = std::max(amax, std::fabs(hp[i]));
-                const float s = block_scale(amax);
+                const float s = block_scale(amax, fmt);
                 rinv = 1.0f / s;
                 scales[((uint64_t)bh * head_elems + s0) / blk] = s;
             }
             for (uint64_t i = s0; i < s0 + blk; ++i) {
                 const uint64_t local = (uint64_t)bh * head_elems + i;
                 const uint64_t flat = (uint64_t)batch_index_base * H * head_elems + local;
-                const float v = (fmt == FMT_E4M3) ? hp[i] * rinv : hp[i];
+                const float v = has_block_scale(fmt) ? hp[i] * rinv : hp[i];
                 const uint32_t U = threshold_u24(rp, flat, step_t);
                 store_code(state, local, fmt, encode(round_on_grid(v, fmt, rule, U), fmt));
             }
@@ -350,18 +374,18 @@ int oracle_state_update(void* state, float* scales, int fmt, uint32_t scale_bloc
 int oracle_quantize_store(const float* src, void* dst_codes, float* dst_scales, uint64_t n_rows, uint32_t row_len,
                           int fmt, uint32_t scale_block, int rule, uint32_t layer, uint32_t weyl_seed,
                           uint32_t weyl_block, uint64_t sr_seed, uint64_t row_index_base, uint32_t step_t) {
-    if (fmt == FMT_E4M3 && (scale_block == 0 || row_len % scale_block != 0 || !dst_scales)) return -1;
+    if (has_block_scale(fmt) && (scale_block == 0 || row_len % scale_block != 0 || !dst_scales)) return -1;
     if (rule == RULE_WEYL && (weyl_block == 0 || row_len % weyl_block != 0)) return -1;
     const RuleParams rp{rule, layer, weyl_seed, weyl_block, sr_seed};
-    const uint32_t blk = (fmt == FMT_E4M3) ? scale_block : row_len;
+    const uint32_t blk = has_block_scale(fmt) ? scale_block : row_len;
 #pragma omp parallel for schedule(static)
     for (int64_t row = 0; row < (int64_t)n_rows; ++row) {
         for (uint32_t s0 = 0; s0 < row_len; s0 += blk) {
             float rinv = 1.0f;
-            if (fmt == FMT_E4M3) {
+            if (has_block_scale(fmt)) {
                 float amax = 0.0f;
                 for (uint32_t i = s0; i < s0 + blk; ++i) amax = std::max(amax, std::fabs(src[(uint64_t)row * row_len + i]));
-                const float s = block_scale(amax);
+                const float s = block_scale(amax, fmt);
                 rinv = 1.0f / s;
                 dst_scales[((uint64_t)row * row_len + s0) / blk] = s;
             }
@@ -369,7 +393,7 @@ int oracle_quantize_store(const float* src, void* dst_codes, float* dst_scales, 
                 const uint64_t local = (uint64_t)row * row_len + i;
                 const uint64_t flat = row_index_base * row_len + local;
                 const float h = src[local];
-                const float v = (fmt == FMT_E4M3) ? h * rinv : h;
+                const float v = has_block_scale(fmt) ? h * rinv : h;
                 const uint32_t U = threshold_u24(rp, flat, step_t);
                 store_code(dst_codes, local, fmt, encode(round_on_grid(v, fmt, rule, U), fmt));
             }
@@ -382,7 +406,7 @@ int oracle_quantize_store(const float* src, void* dst_codes, float* dst_scales, 
 void oracle_dequantize(const void* codes, const float* scales, uint64_t n, int fmt, uint32_t scale_block, float* out) {
     for (uint64_t i = 0; i < n; ++i) {
         float v = decode(load_code(codes, i, fmt), fmt);
-        if (fmt == FMT_E4M3) v = v * scales[i / scale_block];
+        if (has_block_scale(fmt)) v = v * scales[i / scale_block];
         out[i] = v;
     }
 }
