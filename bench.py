@@ -106,7 +106,7 @@ class Stack:
         import torch
         from paper_2609_39185_b200 import ssdq
         self.cfg, self.rule, self.ssdq = cfg, rule, ssdq
-        code_dtype = torch.uint8 if cfg.fmt == workloads.E4M3 else torch.int16
+        code_dtype = torch.uint8 if workloads.CODE_BYTES[cfg.fmt] == 1 else torch.int16
         self.states, self.scales, self.descs, self.keep = [], [], [], []
         for l in range(cfg.n_layers):
             ls = workloads.layer_seed(cfg, seed, l)
@@ -114,7 +114,7 @@ class Stack:
             A_d, D_d = torch.from_numpy(A).cuda(), torch.from_numpy(D).cuda()
             st = torch.zeros(cfg.state_shape, dtype=code_dtype, device="cuda")
             sc = None
-            if cfg.fmt == workloads.E4M3:
+            if cfg.fmt in workloads.SCALED_FORMATS:
                 sc = torch.full((cfg.entries_per_layer // cfg.scale_block,), float(np.finfo(np.float32).tiny),
                                 dtype=torch.float32, device="cuda")
             w = ssdq.weyl_offsets_init(l, 0, cfg.weyl_block)
@@ -234,6 +234,8 @@ def main():
     ap.add_argument("--rule", default="weyl", choices=list(RULE_IDS))
     ap.add_argument("--config", type=int, default=5)
     ap.add_argument("--batch", type=int, default=0, help="override the configuration's batch")
+    ap.add_argument("--format", default="", choices=["", "fp16", "bf16", "e4m3", "int8", "int7", "int6", "int4"],
+                    help="override the configuration's state store format")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling captures)")
     ap.add_argument("--ring", type=int, default=4, help="distinct decode steps of inputs kept resident")
     ap.add_argument("--sweep-batch", default="", help="comma-separated batch sizes: print steps/s per rule for each, then exit")
@@ -244,9 +246,12 @@ def main():
     cfg = workloads.CONFIGS[args.config]
     if args.batch:
         cfg = cfg.with_batch(args.batch)
+    from dataclasses import replace
     if args.layers:
-        from dataclasses import replace
         cfg = replace(cfg, n_layers=args.layers)
+    if args.format:
+        fmt = {v: k for k, v in workloads.FORMAT_NAMES.items()}[args.format]
+        cfg = replace(cfg, fmt=fmt, scale_block=(cfg.scale_block or cfg.weyl_block) if fmt in workloads.SCALED_FORMATS else 0)
     if args.impl == "reference":
         return run_reference(args, cfg)
 
@@ -304,7 +309,7 @@ def main():
             "steps_per_s": args.steps / secs, "pct_of_nominal_8tbs": 100.0 * gbs / world / NOMINAL_HBM_GBS,
             "pct_of_measured_copy": 100.0 * gbs / world / peak,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": None if args.batch else NCU_TRAFFIC_BYTES.get((cfg.index, args.rule)),
+                         "traffic": None if (args.batch or args.format) else NCU_TRAFFIC_BYTES.get((cfg.index, args.rule)),
                          "kernel": "ssd_update_tile_kernel" if cfg.headdim >= 32 and not cfg.a_per_state else "ssd_update_kernel", "peak_source": peak_src,
                          "algorithmic_bytes_per_launch": bytes_per_launch, "launch_us": launch_secs * 1e6},
             "clocks": clocks, "gpu_launches": int(launches)}

@@ -41,7 +41,13 @@ typedef enum {
 
 /* Storage formats (Appendix B "Formats").  SSDQ_FP32 stores binary32 and never rounds: it is the
  * full-precision twin that the quantised trajectory is compared with. */
-typedef enum { SSDQ_FP16 = 0, SSDQ_BF16 = 1, SSDQ_E4M3 = 2, SSDQ_FP32 = 3 } ssdq_format;
+typedef enum {
+    SSDQ_FP16 = 0, SSDQ_BF16 = 1, SSDQ_E4M3 = 2, SSDQ_FP32 = 3,
+    /* Symmetric block-absmax integers (Appendix B "Formats", INTb): one int8 per entry holding k in
+     * [-q_max, q_max], q_max = 2^(b-1) - 1 = 127 / 63 / 31 / 7, value = k * s with the FP32 block scale
+     * s = max(amax_block / q_max, FLT_MIN).  The grid is uniform, so Eq. 2 is floor(v + u) on v = h' * (1/s). */
+    SSDQ_INT8 = 4, SSDQ_INT7 = 5, SSDQ_INT6 = 6, SSDQ_INT4 = 7
+} ssdq_format;
 
 /* Threshold rules of Eq. 2.  RTN rounds to nearest, ties to even (the rule of native casts). */
 typedef enum { SSDQ_RTN = 0, SSDQ_SR_PHILOX = 1, SSDQ_WEYL = 2 } ssdq_rule;
@@ -76,8 +82,8 @@ typedef struct {
     uint32_t batch, nheads, headdim, dstate;  /* B, H, P, N.  N in {16, 32, 64, 128, 256} (E4M3: N >= 16;
                                                  FP32: N >= 16).  Mamba-1 is H = d_inner, P = 1. */
     void* state;         /* [B, H, P, N] codes of `format`, N contiguous, 16-byte aligned; updated IN PLACE */
-    float* scales;       /* E4M3 only: [B, H, P, N / scale_block] FP32 block scales, updated in place */
-    uint32_t scale_block;/* E4M3 only: 16 or N (entries along N that share one scale) */
+    float* scales;       /* E4M3 and INTb: [B, H, P, N / scale_block] FP32 block scales, updated in place */
+    uint32_t scale_block;/* E4M3 and INTb: 16 or N (entries along N that share one scale) */
     int32_t format;      /* ssdq_format */
     const float* x;      /* [B, H, P] */
     const float* dt;     /* [B, H], already passed through softplus */
@@ -98,7 +104,7 @@ typedef struct {
  *   h  = dequant(state)                          (E4M3: code * scale, one rounded multiply)
  *   a  = exp_spec(dt*A);  w = (dt*x)*B;  h' = fma(a, h, w)      all binary32, in this order
  *   y  = sum_n C[n]*h'[n] + D*x                  (FP32 accumulation, tree order unspecified)
- *   E4M3: s = max(amax_block(h') / 448, FLT_MIN), v = h' * (1/s);  otherwise v = h'
+ *   E4M3 / INTb: s = max(amax_block(h') / top, FLT_MIN) with top = 448 / q_max, v = h' * (1/s);  otherwise v = h'
  *   state = encode(Q_u(v)) with u from `rule` at write index step_t (first write is step_t = 1)
  * exp_spec is the library's fixed binary32 exponential (clamp to [-87, 88], Cody-Waite reduction,
  * degree-7 polynomial), identical bit for bit on every call.  Values beyond the format's largest

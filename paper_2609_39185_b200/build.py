@@ -16,7 +16,7 @@ ROOT = os.path.dirname(HERE)
 LIB = os.path.join(HERE, "libssdq.so")
 OBJ_DIR = os.path.join(HERE, "build")
 
-SOURCES = ["ssdq_api.cu", "ssdq_update_fp16.cu", "ssdq_update_bf16.cu", "ssdq_update_e4m3.cu", "ssdq_update_fp32.cu",
+SOURCES = ["ssdq_api.cu", "ssdq_update_fp16.cu", "ssdq_update_bf16.cu", "ssdq_update_e4m3.cu", "ssdq_update_fp32.cu", "ssdq_update_int8.cu",
            "ssdq_quantize.cu", "ssdq_metrics.cu"]
 # --fmad=false: nothing is contracted behind the kernels' backs; every fused multiply-add is written out.
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo", "--fmad=false",

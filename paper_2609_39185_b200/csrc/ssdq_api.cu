@@ -31,6 +31,21 @@ int cuda_result(cudaError_t e, const char* what) {
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
 
+bool format_known(int fmt) { return fmt >= SSDQ_FP16 && fmt <= SSDQ_INT4; }
+bool format_scaled(int fmt) { return fmt == SSDQ_E4M3 || (fmt >= SSDQ_INT8 && fmt <= SSDQ_INT4); }
+// kernel family of a public format id, and the top of its scaled range (amax maps onto it)
+int kernel_format(int fmt) { return fmt >= SSDQ_INT8 ? (int)ssdq::FMT_INT : fmt; }
+float scale_top(int fmt) {
+    switch (fmt) {
+        case SSDQ_E4M3: return 448.0f;
+        case SSDQ_INT8: return 127.0f;
+        case SSDQ_INT7: return 63.0f;
+        case SSDQ_INT6: return 31.0f;
+        case SSDQ_INT4: return 7.0f;
+        default: return 1.0f;
+    }
+}
+
 bool dstate_supported(int fmt, uint32_t n) {
     if (!(n == 16 || n == 32 || n == 64 || n == 128 || n == 256)) return false;
     if (fmt == SSDQ_FP32 && n > 128) return false;   // a row of 256 floats would span two warps
@@ -45,7 +60,7 @@ ssdq::WeylConst weyl_const(const ssdq_weyl& w) {
 int check_layer(const ssdq_update_desc* d) {
     if (!d) return fail(SSDQ_ERR_NULL, "descriptor is NULL");
     if (d->batch == 0 || d->nheads == 0 || d->headdim == 0) return fail(SSDQ_ERR_SHAPE, "batch, nheads and headdim must be positive");
-    if (d->format < SSDQ_FP16 || d->format > SSDQ_FP32) return fail(SSDQ_ERR_UNSUPPORTED, "unknown format %d", d->format);
+    if (!format_known(d->format)) return fail(SSDQ_ERR_UNSUPPORTED, "unknown format %d", d->format);
     if (d->rule < SSDQ_RTN || d->rule > SSDQ_WEYL) return fail(SSDQ_ERR_UNSUPPORTED, "unknown rule %d", d->rule);
     if (!dstate_supported(d->format, d->dstate)) return fail(SSDQ_ERR_UNSUPPORTED, "dstate %u is not supported for format %d", d->dstate, d->format);
     if ((uint64_t)d->batch * d->nheads > 0xFFFFFFFFull / 2) return fail(SSDQ_ERR_SHAPE, "batch * nheads too large");
@@ -53,8 +68,8 @@ int check_layer(const ssdq_update_desc* d) {
     if (!aligned16(d->state)) return fail(SSDQ_ERR_ALIGN, "state must be 16-byte aligned");
     if (d->a_per_state ? !aligned16(d->A) : !aligned4(d->A)) return fail(SSDQ_ERR_ALIGN, "A is misaligned");
     if (d->D && !aligned4(d->D)) return fail(SSDQ_ERR_ALIGN, "D is misaligned");
-    if (d->format == SSDQ_E4M3) {
-        if (!d->scales) return fail(SSDQ_ERR_NULL, "E4M3 needs a scale array");
+    if (format_scaled(d->format)) {
+        if (!d->scales) return fail(SSDQ_ERR_NULL, "E4M3 and INTb stores need a scale array");
         if (!aligned4(d->scales)) return fail(SSDQ_ERR_ALIGN, "scales are misaligned");
         if (d->scale_block == (uint32_t)d->headdim * d->dstate && d->scale_block != d->dstate)
             return fail(SSDQ_ERR_UNSUPPORTED, "one scale per head is not built; use scale_block 16 or dstate");
@@ -81,6 +96,7 @@ ssdq::UpdateParams make_params(const ssdq_update_desc* d, uint32_t step_t) {
     p.B = d->batch; p.H = d->nheads; p.P = d->headdim; p.N = d->dstate;
     p.n_items = d->batch * d->nheads;
     p.scale_block = d->scale_block;
+    p.scale_top = scale_top(d->format);
     p.step_t = step_t; p.layer = d->layer; p.batch_base = d->batch_index_base;
     p.weyl = weyl_const(d->weyl);
     p.sr_seed = d->sr_seed;
@@ -93,6 +109,7 @@ cudaError_t launch_update(const ssdq::UpdateParams& p, int fmt, int rule, bool a
         case SSDQ_BF16: return ssdq::launch_update_bf16(p, rule, aps, s);
         case SSDQ_E4M3: return ssdq::launch_update_e4m3(p, rule, aps, s);
         case SSDQ_FP32: return ssdq::launch_update_fp32(p, rule, aps, s);
+        case SSDQ_INT8: case SSDQ_INT7: case SSDQ_INT6: case SSDQ_INT4: return ssdq::launch_update_int8(p, rule, aps, s);
         default: return cudaErrorInvalidValue;
     }
 }
@@ -191,15 +208,15 @@ int ssd_state_update(const ssdq_update_desc* d, uint32_t step_t, void* stream) {
 int quantize_store(const float* src, void* dst_codes, float* dst_scales, uint64_t n_rows, uint32_t row_len,
                    uint32_t scale_block, int format, int rule, const ssdq_weyl* weyl, uint64_t sr_seed, uint32_t layer,
                    uint64_t row_index_base, uint32_t step_t, void* stream) {
-    if (format < SSDQ_FP16 || format > SSDQ_FP32) return fail(SSDQ_ERR_UNSUPPORTED, "unknown format %d", format);
+    if (!format_known(format)) return fail(SSDQ_ERR_UNSUPPORTED, "unknown format %d", format);
     if (rule < SSDQ_RTN || rule > SSDQ_WEYL) return fail(SSDQ_ERR_UNSUPPORTED, "unknown rule %d", rule);
     if (!dstate_supported(format, row_len)) return fail(SSDQ_ERR_UNSUPPORTED, "row_len %u is not supported for format %d", row_len, format);
     if (n_rows == 0) return SSDQ_OK;
     if (!src || !dst_codes) return fail(SSDQ_ERR_NULL, "src and dst_codes are required");
     if (!aligned16(src) || !aligned16(dst_codes)) return fail(SSDQ_ERR_ALIGN, "src and dst_codes must be 16-byte aligned");
     ssdq::QuantParams p{};
-    if (format == SSDQ_E4M3) {
-        if (!dst_scales) return fail(SSDQ_ERR_NULL, "E4M3 needs a scale array");
+    if (format_scaled(format)) {
+        if (!dst_scales) return fail(SSDQ_ERR_NULL, "E4M3 and INTb stores need a scale array");
         if (!(scale_block == 16 || scale_block == row_len)) return fail(SSDQ_ERR_SHAPE, "scale_block must be 16 or row_len");
     }
     if (rule == SSDQ_WEYL && format != SSDQ_FP32) {
@@ -208,20 +225,20 @@ int quantize_store(const float* src, void* dst_codes, float* dst_scales, uint64_
         p.weyl = weyl_const(*weyl);
     }
     p.src = src; p.codes = dst_codes; p.scales = dst_scales; p.n_rows = n_rows; p.row_len = row_len;
-    p.scale_block = scale_block; p.step_t = step_t; p.layer = layer; p.row_base = row_index_base; p.sr_seed = sr_seed;
-    return cuda_result(ssdq::launch_quantize(p, format, rule, static_cast<cudaStream_t>(stream)), "quantize kernel");
+    p.scale_block = scale_block; p.scale_top = scale_top(format); p.step_t = step_t; p.layer = layer; p.row_base = row_index_base; p.sr_seed = sr_seed;
+    return cuda_result(ssdq::launch_quantize(p, kernel_format(format), rule, static_cast<cudaStream_t>(stream)), "quantize kernel");
 }
 
 int ssdq_dequantize(const void* codes, const float* scales, uint64_t n, int format, uint32_t scale_block, float* out,
                     void* stream) {
-    if (format < SSDQ_FP16 || format > SSDQ_FP32) return fail(SSDQ_ERR_UNSUPPORTED, "unknown format %d", format);
+    if (!format_known(format)) return fail(SSDQ_ERR_UNSUPPORTED, "unknown format %d", format);
     if (n == 0) return SSDQ_OK;
     if (!codes || !out) return fail(SSDQ_ERR_NULL, "codes and out are required");
     if (n % 16 != 0) return fail(SSDQ_ERR_SHAPE, "n must be a multiple of 16");
     if (!aligned16(codes) || !aligned16(out)) return fail(SSDQ_ERR_ALIGN, "codes and out must be 16-byte aligned");
-    if (format == SSDQ_E4M3 && (!scales || scale_block == 0 || scale_block % 16 != 0))
-        return fail(SSDQ_ERR_SHAPE, "E4M3 needs scales and a scale_block that is a multiple of 16");
-    return cuda_result(ssdq::launch_dequantize(codes, scales, n, format, scale_block, out, static_cast<cudaStream_t>(stream)),
+    if (format_scaled(format) && (!scales || scale_block == 0 || scale_block % 16 != 0))
+        return fail(SSDQ_ERR_SHAPE, "scaled stores need scales and a scale_block that is a multiple of 16");
+    return cuda_result(ssdq::launch_dequantize(codes, scales, n, kernel_format(format), scale_block, out, static_cast<cudaStream_t>(stream)),
                        "dequantize kernel");
 }
 
@@ -266,16 +283,16 @@ uint64_t ssdq_state_error_workspace_bytes(uint32_t batch, uint32_t nheads) { ret
 int ssdq_state_error(const void* codes, const float* scales, const float* twin, uint32_t batch, uint32_t nheads,
                      uint32_t headdim, uint32_t dstate, int format, uint32_t scale_block, double* err2_per_head,
                      double* ref2_per_head, void* workspace, uint64_t workspace_bytes, void* stream) {
-    if (format < SSDQ_FP16 || format > SSDQ_FP32) return fail(SSDQ_ERR_UNSUPPORTED, "unknown format %d", format);
+    if (!format_known(format)) return fail(SSDQ_ERR_UNSUPPORTED, "unknown format %d", format);
     if (batch == 0 || nheads == 0 || headdim == 0 || dstate == 0) return fail(SSDQ_ERR_SHAPE, "sizes must be positive");
     if (((uint64_t)headdim * dstate) % 16 != 0) return fail(SSDQ_ERR_SHAPE, "headdim * dstate must be a multiple of 16");
     if ((uint64_t)batch * nheads > 0x7FFFFFFFull) return fail(SSDQ_ERR_SHAPE, "batch * nheads too large");
     if (!codes || !twin || !err2_per_head || !ref2_per_head || !workspace) return fail(SSDQ_ERR_NULL, "codes, twin, outputs and workspace are required");
     if (!aligned16(codes) || !aligned16(workspace) || !aligned4(twin)) return fail(SSDQ_ERR_ALIGN, "codes and workspace must be 16-byte aligned");
     if (workspace_bytes < ssdq_state_error_workspace_bytes(batch, nheads)) return fail(SSDQ_ERR_SHAPE, "workspace too small");
-    if (format == SSDQ_E4M3 && (!scales || scale_block == 0 || scale_block % 16 != 0))
-        return fail(SSDQ_ERR_SHAPE, "E4M3 needs scales and a scale_block that is a multiple of 16");
-    const int rc = cuda_result(ssdq::launch_state_error(codes, scales, twin, batch, nheads, headdim * dstate, format, scale_block,
+    if (format_scaled(format) && (!scales || scale_block == 0 || scale_block % 16 != 0))
+        return fail(SSDQ_ERR_SHAPE, "scaled stores need scales and a scale_block that is a multiple of 16");
+    const int rc = cuda_result(ssdq::launch_state_error(codes, scales, twin, batch, nheads, headdim * dstate, kernel_format(format), scale_block,
                                                         err2_per_head, ref2_per_head, workspace, static_cast<cudaStream_t>(stream)),
                                "state-error kernels");
     if (rc == SSDQ_OK) g_launches.fetch_add(1, std::memory_order_relaxed);   // two kernels per call

@@ -19,7 +19,8 @@ struct UpdateParams {
     float* y;
     uint32_t B, H, P, N;
     uint32_t n_items;        // B * H
-    uint32_t scale_block;    // E4M3: 16 or N
+    uint32_t scale_block;    // scaled stores: 16 or N
+    float scale_top;         // scaled stores: block scale = amax / scale_top (448 for E4M3, q_max for INTb)
     uint32_t step_t;
     uint32_t layer;
     uint32_t batch_base;
@@ -38,6 +39,7 @@ struct QuantParams {
     uint64_t n_rows;
     uint32_t row_len;
     uint32_t scale_block;
+    float scale_top;
     uint32_t step_t;
     uint32_t layer;
     uint64_t row_base;
@@ -50,6 +52,7 @@ cudaError_t launch_update_fp16(const UpdateParams& p, int rule, bool a_per_state
 cudaError_t launch_update_bf16(const UpdateParams& p, int rule, bool a_per_state, cudaStream_t s);
 cudaError_t launch_update_e4m3(const UpdateParams& p, int rule, bool a_per_state, cudaStream_t s);
 cudaError_t launch_update_fp32(const UpdateParams& p, int rule, bool a_per_state, cudaStream_t s);
+cudaError_t launch_update_int8(const UpdateParams& p, int rule, bool a_per_state, cudaStream_t s);
 
 cudaError_t launch_quantize(const QuantParams& p, int fmt, int rule, cudaStream_t s);
 cudaError_t launch_dequantize(const void* codes, const float* scales, uint64_t n, int fmt, uint32_t scale_block,

@@ -39,7 +39,7 @@ __global__ void __launch_bounds__(kMetricThreads) state_error_partial_kernel(con
     for (uint32_t i = threadIdx.x * EPL; i < item_elems; i += kMetricThreads * EPL) {
         float h[EPL];
         unpack_lane<FMT>(codes[(first + i) / EPL], h);
-        if constexpr (FMT == FMT_E4M3) {
+        if constexpr (Fmt<FMT>::kScaled) {
             const float s = scales[(first + i) / scale_block];
 #pragma unroll
             for (int j = 0; j < EPL; ++j) h[j] = __fmul_rn(h[j], s);
@@ -82,6 +82,7 @@ cudaError_t launch_state_error(const void* codes, const float* scales, const flo
         case FMT_FP16: state_error_partial_kernel<FMT_FP16><<<n_items, kMetricThreads, 0, s>>>(c, scales, twin, item_elems, scale_block, partial); break;
         case FMT_BF16: state_error_partial_kernel<FMT_BF16><<<n_items, kMetricThreads, 0, s>>>(c, scales, twin, item_elems, scale_block, partial); break;
         case FMT_E4M3: state_error_partial_kernel<FMT_E4M3><<<n_items, kMetricThreads, 0, s>>>(c, scales, twin, item_elems, scale_block, partial); break;
+        case FMT_INT: state_error_partial_kernel<FMT_INT><<<n_items, kMetricThreads, 0, s>>>(c, scales, twin, item_elems, scale_block, partial); break;
         case FMT_FP32: state_error_partial_kernel<FMT_FP32><<<n_items, kMetricThreads, 0, s>>>(c, scales, twin, item_elems, scale_block, partial); break;
         default: return cudaErrorInvalidValue;
     }
@@ -167,7 +168,7 @@ int static_scratch_for_current_device(double2** out) {
 extern "C" int ssdq_state_error_static(const void* codes, const float* scales, const float* twin, uint32_t batch,
                                        uint32_t nheads, uint32_t headdim, uint32_t dstate, int format,
                                        uint32_t scale_block, double* err2_per_head, double* ref2_per_head, void* stream) {
-    if (format < SSDQ_FP16 || format > SSDQ_FP32) return ssdq::report_failure(SSDQ_ERR_UNSUPPORTED, "unknown format");
+    if (format < SSDQ_FP16 || format > SSDQ_INT4) return ssdq::report_failure(SSDQ_ERR_UNSUPPORTED, "unknown format");
     if (batch == 0 || nheads == 0 || headdim == 0 || dstate == 0) return ssdq::report_failure(SSDQ_ERR_SHAPE, "sizes must be positive");
     if (((uint64_t)headdim * dstate) % 16 != 0) return ssdq::report_failure(SSDQ_ERR_SHAPE, "headdim * dstate must be a multiple of 16");
     if ((uint64_t)batch * nheads > kStaticMaxItems)
@@ -176,13 +177,15 @@ extern "C" int ssdq_state_error_static(const void* codes, const float* scales, c
     if (!codes || !twin || !err2_per_head || !ref2_per_head) return ssdq::report_failure(SSDQ_ERR_NULL, "codes, twin and outputs are required");
     if ((reinterpret_cast<uintptr_t>(codes) & 15u) || (reinterpret_cast<uintptr_t>(twin) & 3u))
         return ssdq::report_failure(SSDQ_ERR_ALIGN, "codes must be 16-byte aligned");
-    if (format == SSDQ_E4M3 && (!scales || scale_block == 0 || scale_block % 16 != 0))
-        return ssdq::report_failure(SSDQ_ERR_SHAPE, "E4M3 needs scales and a scale_block that is a multiple of 16");
+    const bool scaled = format == SSDQ_E4M3 || format >= SSDQ_INT8;
+    if (scaled && (!scales || scale_block == 0 || scale_block % 16 != 0))
+        return ssdq::report_failure(SSDQ_ERR_SHAPE, "scaled stores need scales and a scale_block that is a multiple of 16");
     double2* scratch = nullptr;
     const int rc = static_scratch_for_current_device(&scratch);
     if (rc != SSDQ_OK) return rc;
     // every partial the second pass reads is written by the first pass of this same call: nothing has to be cleared
-    const cudaError_t e = ssdq::launch_state_error(codes, scales, twin, batch, nheads, headdim * dstate, format, scale_block,
+    const cudaError_t e = ssdq::launch_state_error(codes, scales, twin, batch, nheads, headdim * dstate,
+                                                   format >= SSDQ_INT8 ? (int)ssdq::FMT_INT : format, scale_block,
                                                    err2_per_head, ref2_per_head, scratch, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return ssdq::report_failure(SSDQ_ERR_CUDA, cudaGetErrorString(e));
     ssdq::count_launches(2);

@@ -16,7 +16,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantParams p)
     LaneThreshold<FMT, RULE, LPR> thr;
     thr.init(p.weyl, p.step_t, lis);
     const uint32_t key0 = (uint32_t)p.sr_seed, key1 = (uint32_t)(p.sr_seed >> 32);
-    const bool row_scale = (FMT == FMT_E4M3) && (p.scale_block == (uint32_t)N);
+    const bool row_scale = Fmt<FMT>::kScaled && (p.scale_block == (uint32_t)N);
     const uint64_t rows_per_pass = (uint64_t)gridDim.x * NSLOT;
     const uint64_t n_pass = (p.n_rows + rows_per_pass - 1) / rows_per_pass;    // uniform trip count: shuffles inside
     for (uint64_t it = 0; it < n_pass; ++it) {
@@ -29,7 +29,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantParams p)
             if (ok) f = reinterpret_cast<const float4*>(p.src + row * N + lis * EPL)[i];
             v[4 * i] = f.x; v[4 * i + 1] = f.y; v[4 * i + 2] = f.z; v[4 * i + 3] = f.w;
         }
-        if constexpr (FMT == FMT_E4M3) {
+        if constexpr (Fmt<FMT>::kScaled) {
             float amax = 0.0f;
 #pragma unroll
             for (int j = 0; j < EPL; ++j) amax = fmaxf(amax, fabsf(v[j]));
@@ -37,7 +37,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantParams p)
 #pragma unroll
                 for (int off = LPR / 2; off > 0; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, off));
             }
-            const float s = fmaxf(__fdiv_rn(amax, 448.0f), 1.17549435e-38f);
+            const float s = fmaxf(__fdiv_rn(amax, p.scale_top), 1.17549435e-38f);
             const float rinv = __fdiv_rn(1.0f, s);
 #pragma unroll
             for (int j = 0; j < EPL; ++j) v[j] = __fmul_rn(v[j], rinv);
@@ -50,7 +50,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantParams p)
         uint32_t g_lo = 0, g_hi = 0, acc0 = 0;
         if constexpr (RULE == RULE_WEYL) acc0 = thr.weyl_acc0(grow);
         if constexpr (RULE == RULE_SR) thr.sr_group(grow, g_lo, g_hi);
-        const uint4 packed = round_pack_lane<FMT, RULE>(v, acc0, p.weyl.mul_col, g_lo, g_hi, p.step_t, p.layer, key0, key1);
+        const uint4 packed = round_pack_lane<FMT, RULE>(v, acc0, p.weyl.mul_col, g_lo, g_hi, p.step_t, p.layer, key0, key1, p.scale_top);
         if (ok) reinterpret_cast<uint4*>(p.codes)[row * LPR + lis] = packed;
     }
 }
@@ -96,6 +96,7 @@ cudaError_t launch_quantize(const QuantParams& p, int fmt, int rule, cudaStream_
         case FMT_FP16: return launch_quantize_fmt<FMT_FP16>(p, rule, s);
         case FMT_BF16: return launch_quantize_fmt<FMT_BF16>(p, rule, s);
         case FMT_E4M3: return launch_quantize_fmt<FMT_E4M3>(p, rule, s);
+        case FMT_INT: return launch_quantize_fmt<FMT_INT>(p, rule, s);
         case FMT_FP32: return launch_quantize_n<FMT_FP32, RULE_RTN>(p, s);
         default: return cudaErrorInvalidValue;
     }
@@ -109,7 +110,7 @@ __global__ void __launch_bounds__(256) dequantize_kernel(const uint4* __restrict
     for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec; i += (uint64_t)gridDim.x * blockDim.x) {
         float h[EPL];
         unpack_lane<FMT>(codes[i], h);
-        if constexpr (FMT == FMT_E4M3) {
+        if constexpr (Fmt<FMT>::kScaled) {
             const float s = scales[(i * EPL) / scale_block];     // 16 consecutive entries share a scale
 #pragma unroll
             for (int j = 0; j < EPL; ++j) h[j] = __fmul_rn(h[j], s);
@@ -129,6 +130,7 @@ cudaError_t launch_dequantize(const void* codes, const float* scales, uint64_t n
         case FMT_FP16: dequantize_kernel<FMT_FP16><<<grid_of(n / 8), 256, 0, s>>>(c, scales, n / 8, scale_block, out); break;
         case FMT_BF16: dequantize_kernel<FMT_BF16><<<grid_of(n / 8), 256, 0, s>>>(c, scales, n / 8, scale_block, out); break;
         case FMT_E4M3: dequantize_kernel<FMT_E4M3><<<grid_of(n / 16), 256, 0, s>>>(c, scales, n / 16, scale_block, out); break;
+        case FMT_INT: dequantize_kernel<FMT_INT><<<grid_of(n / 16), 256, 0, s>>>(c, scales, n / 16, scale_block, out); break;
         case FMT_FP32: dequantize_kernel<FMT_FP32><<<grid_of(n / 4), 256, 0, s>>>(c, scales, n / 4, scale_block, out); break;
         default: return cudaErrorInvalidValue;
     }

@@ -19,6 +19,7 @@ constexpr int kThreads = 128;
 
 template <int FMT> struct Unroll { static constexpr int value = 4; };
 template <> struct Unroll<FMT_E4M3> { static constexpr int value = 2; };
+template <> struct Unroll<FMT_INT> { static constexpr int value = 2; };
 
 // Unpack the lane's 16 bytes into EPL floats (exact widening; E4M3 is multiplied by its scale later).
 template <int FMT>
@@ -33,6 +34,9 @@ __device__ __forceinline__ void unpack_lane(const uint4& raw, float* h) {
     } else if constexpr (FMT == FMT_E4M3) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) unpack4_e4m3(w[i], h + 4 * i);
+    } else if constexpr (FMT == FMT_INT) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) unpack4_int8(w[i], h + 4 * i);
     } else {
 #pragma unroll
         for (int i = 0; i < 4; ++i) h[i] = __uint_as_float(w[i]);
@@ -45,7 +49,7 @@ __device__ __forceinline__ void unpack_lane(const uint4& raw, float* h) {
 template <int FMT, int RULE>
 __device__ __forceinline__ uint4 round_pack_lane(const float* v, uint32_t acc0, uint32_t mul_col, uint32_t g_lo,
                                                  uint32_t g_hi, uint32_t step_t, uint32_t layer, uint32_t key0,
-                                                 uint32_t key1) {
+                                                 uint32_t key1, float qmax) {
     constexpr int EPL = Fmt<FMT>::kEpl;
     uint32_t w[4];
     if constexpr (FMT == FMT_FP32) {
@@ -58,6 +62,11 @@ __device__ __forceinline__ uint4 round_pack_lane(const float* v, uint32_t acc0, 
         } else if constexpr (FMT == FMT_BF16) {
 #pragma unroll
             for (int i = 0; i < 4; ++i) w[i] = rtn_pack2_bf16(v[2 * i], v[2 * i + 1]);
+        } else if constexpr (FMT == FMT_INT) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                w[i] = pack4_low_bytes(int_rtn_biased(v[4 * i], qmax), int_rtn_biased(v[4 * i + 1], qmax),
+                                       int_rtn_biased(v[4 * i + 2], qmax), int_rtn_biased(v[4 * i + 3], qmax));
         } else {
 #pragma unroll
             for (int i = 0; i < 4; ++i)
@@ -102,6 +111,11 @@ __device__ __forceinline__ uint4 round_pack_lane(const float* v, uint32_t acc0, 
                 }
                 w[i] = rtn_pack2_fp16(r[0], r[1]);   // exact: r is on the FP16 grid; saturates beyond 65504
             }
+        } else if constexpr (FMT == FMT_INT) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                w[i] = pack4_low_bytes(int_dither_biased(v[4 * i], acc[4 * i], qmax), int_dither_biased(v[4 * i + 1], acc[4 * i + 1], qmax),
+                                       int_dither_biased(v[4 * i + 2], acc[4 * i + 2], qmax), int_dither_biased(v[4 * i + 3], acc[4 * i + 3], qmax));
         } else {
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -205,7 +219,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_kernel(const UpdateParams
     const uint64_t row_first = (uint64_t)item * p.P + p_first;    // local row index (this call's tensors)
     const uint64_t grow_first = row_first + (uint64_t)p.batch_base * p.H * p.P;   // global row index
     uint4* state = reinterpret_cast<uint4*>(p.state);
-    const bool row_scale = (FMT == FMT_E4M3) && (p.scale_block == (uint32_t)N);
+    const bool row_scale = Fmt<FMT>::kScaled && (p.scale_block == (uint32_t)N);
 
     float ykeep = 0.0f;
     for (uint32_t k0 = 0; k0 < p.rps; k0 += UNR) {
@@ -224,7 +238,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_kernel(const UpdateParams
                 const uint64_t row = row_first + k;
                 raw[u] = state[row * LPR + lis];
                 xv[u] = __ldg(p.x + row);
-                if constexpr (FMT == FMT_E4M3)
+                if constexpr (Fmt<FMT>::kScaled)
                     sc[u] = row_scale ? p.scales[row] : p.scales[row * (N / 16) + lis];
             }
         }
@@ -240,22 +254,22 @@ __global__ void __launch_bounds__(kThreads) ssd_update_kernel(const UpdateParams
 #pragma unroll
             for (int j = 0; j < EPL; ++j) {
                 float hin = hv[j];
-                if constexpr (FMT == FMT_E4M3) hin = __fmul_rn(hin, sc[u]);
+                if constexpr (Fmt<FMT>::kScaled) hin = __fmul_rn(hin, sc[u]);
                 const float w = __fmul_rn(dtx, Bv[j]);
                 const float hn = __fmaf_rn(APS ? av[APS ? j : 0] : av[0], hin, w);
                 hv[j] = hn;
                 dot = __fmaf_rn(Cv[j], hn, dot);
-                if constexpr (FMT == FMT_E4M3) amax = fmaxf(amax, fabsf(hn));
+                if constexpr (Fmt<FMT>::kScaled) amax = fmaxf(amax, fabsf(hn));
             }
             // readout: reduce the partial dots over the slot
 #pragma unroll
             for (int off = LPR / 2; off > 0; off >>= 1) dot += __shfl_xor_sync(FULL, dot, off);
-            if constexpr (FMT == FMT_E4M3) {
+            if constexpr (Fmt<FMT>::kScaled) {
                 if (row_scale) {
 #pragma unroll
                     for (int off = LPR / 2; off > 0; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, off));
                 }
-                const float s = fmaxf(__fdiv_rn(amax, 448.0f), 1.17549435e-38f);
+                const float s = fmaxf(__fdiv_rn(amax, p.scale_top), 1.17549435e-38f);
                 const float rinv = __fdiv_rn(1.0f, s);
 #pragma unroll
                 for (int j = 0; j < EPL; ++j) hv[j] = __fmul_rn(hv[j], rinv);
@@ -268,7 +282,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_kernel(const UpdateParams
             if constexpr (RULE == RULE_WEYL) acc0 = thr.weyl_acc0(grow_first + k);
             if constexpr (RULE == RULE_SR) thr.sr_group(grow_first + k, g_lo, g_hi);
             const uint4 packed = round_pack_lane<FMT, RULE>(hv, acc0, p.weyl.mul_col, g_lo, g_hi, p.step_t, p.layer,
-                                                             key0, key1);
+                                                             key0, key1, p.scale_top);
             if (ok[u]) state[row * LPR + lis] = packed;
             // y: lane (k mod LPR) of the slot keeps row k; flushed every LPR rows
             const float yv = __fmaf_rn(Dv, xv[u], dot);
@@ -323,7 +337,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
     const uint32_t h = item - b * p.H;
     const uint32_t n0 = lis * EPL;
     const uint64_t row_first = (uint64_t)item * (NSLOT * RPS) + slot * RPS;
-    const bool row_scale = (FMT == FMT_E4M3) && (p.scale_block == (uint32_t)N);
+    const bool row_scale = Fmt<FMT>::kScaled && (p.scale_block == (uint32_t)N);
 
     // every load of the CTA is issued here
     uint4* sp = reinterpret_cast<uint4*>(p.state) + row_first * LPR + lis;
@@ -331,13 +345,13 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
 #pragma unroll
     for (int k = 0; k < RPS; ++k) raw[k] = sp[k * LPR];
     float xv[RPS];
-    float sc[FMT == FMT_E4M3 ? RPS : 1];
+    float sc[Fmt<FMT>::kScaled ? RPS : 1];
 #pragma unroll
     for (int k = 0; k < RPS / 4; ++k) {
         const float4 x4 = __ldg(reinterpret_cast<const float4*>(p.x + row_first) + k);
         xv[4 * k] = x4.x; xv[4 * k + 1] = x4.y; xv[4 * k + 2] = x4.z; xv[4 * k + 3] = x4.w;
     }
-    if constexpr (FMT == FMT_E4M3) {
+    if constexpr (Fmt<FMT>::kScaled) {
 #pragma unroll
         for (int k = 0; k < RPS; ++k) sc[k] = row_scale ? p.scales[row_first + k] : p.scales[(row_first + k) * (N / 16) + lis];
     }
@@ -379,19 +393,19 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
 #pragma unroll
             for (int j = 0; j < EPL; ++j) {
                 float hin = hv[j];
-                if constexpr (FMT == FMT_E4M3) hin = __fmul_rn(hin, sc[k]);
+                if constexpr (Fmt<FMT>::kScaled) hin = __fmul_rn(hin, sc[k]);
                 const float hn = __fmaf_rn(a, hin, __fmul_rn(dtx, Bv[j]));
                 hv[j] = hn;
                 dot = __fmaf_rn(Cv[j], hn, dot);
-                if constexpr (FMT == FMT_E4M3) amax = fmaxf(amax, fabsf(hn));
+                if constexpr (Fmt<FMT>::kScaled) amax = fmaxf(amax, fabsf(hn));
             }
             dots[u] = dot;
-            if constexpr (FMT == FMT_E4M3) {
+            if constexpr (Fmt<FMT>::kScaled) {
                 if (row_scale) {
 #pragma unroll
                     for (int off = LPR / 2; off > 0; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, off));
                 }
-                const float s = fmaxf(__fdiv_rn(amax, 448.0f), 1.17549435e-38f);
+                const float s = fmaxf(__fdiv_rn(amax, p.scale_top), 1.17549435e-38f);
                 const float rinv = __fdiv_rn(1.0f, s);
 #pragma unroll
                 for (int j = 0; j < EPL; ++j) hv[j] = __fmul_rn(hv[j], rinv);
@@ -399,7 +413,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
                 else p.scales[(row_first + k) * (N / 16) + lis] = s;
             }
             const uint4 packed = round_pack_lane<FMT, RULE>(hv, acc_row, p.weyl.mul_col, (uint32_t)grp_row,
-                                                             (uint32_t)(grp_row >> 32), p.step_t, p.layer, key0, key1);
+                                                             (uint32_t)(grp_row >> 32), p.step_t, p.layer, key0, key1, p.scale_top);
             sp[k * LPR] = packed;
             if constexpr (RULE == RULE_WEYL) acc_row += thr.row_mul;
             if constexpr (RULE == RULE_SR) grp_row += N / 4;
@@ -417,7 +431,7 @@ inline cudaError_t launch_update_one(const UpdateParams& p, cudaStream_t stream)
     if constexpr (!APS && LPR >= 4 && FMT != FMT_FP32) {
         // shapes the tile kernel covers: a head of nslot * {4, 8} rows; x, y (and row scales) 16-byte aligned
         const bool aligned = ((reinterpret_cast<uintptr_t>(q.x) | reinterpret_cast<uintptr_t>(q.y)) & 15u) == 0 &&
-                             (FMT != FMT_E4M3 || (reinterpret_cast<uintptr_t>(q.scales) & 15u) == 0);
+                             (!Fmt<FMT>::kScaled || (reinterpret_cast<uintptr_t>(q.scales) & 15u) == 0);
         if (aligned && q.P == nslot * 8u) {
             ssd_update_tile_kernel<FMT, RULE, LPR, 8><<<q.n_items, kThreads, 0, stream>>>(q);
             return cudaGetLastError();

@@ -36,12 +36,12 @@ def run(cfg, steps, log_every, chunk=128, seed=0, layer=0, emit=print):
     from . import ssdq
     A, D = workloads.layer_params(cfg, layer, seed)
     A_d, D_d = torch.from_numpy(A).cuda(), torch.from_numpy(D).cuda()
-    code_dtype = torch.uint8 if cfg.fmt == workloads.E4M3 else torch.int16
+    code_dtype = torch.uint8 if workloads.CODE_BYTES[cfg.fmt] == 1 else torch.int16
     runs = {}
     for name, rid in RULES:
         st = torch.zeros(cfg.state_shape, dtype=code_dtype, device="cuda")
         sc = None
-        if cfg.fmt == workloads.E4M3:
+        if cfg.fmt in workloads.SCALED_FORMATS:
             sc = torch.full((cfg.entries_per_layer // cfg.scale_block,), float(np.finfo(np.float32).tiny),
                             dtype=torch.float32, device="cuda")
         desc = ssdq.make_desc(st, sc, cfg.fmt, A=A_d, D=D_d, rule=rid, weyl=ssdq.weyl_offsets_init(layer, 0, cfg.weyl_block),
@@ -89,12 +89,16 @@ def main():
     ap.add_argument("--steps", type=int, default=0)
     ap.add_argument("--log-every", type=int, default=256)
     ap.add_argument("--batch", type=int, default=0)
+    ap.add_argument("--format", default="", choices=["", "fp16", "bf16", "e4m3", "int8", "int7", "int6", "int4"])
     ap.add_argument("--out", default="")
     args = ap.parse_args()
     cfg = workloads.CONFIGS[args.config]
     if args.batch:
         cfg = cfg.with_batch(args.batch)
     cfg = replace(cfg, n_layers=1)
+    if args.format:
+        fmt = {v: k for k, v in workloads.FORMAT_NAMES.items()}[args.format]
+        cfg = replace(cfg, fmt=fmt, scale_block=(cfg.scale_block or cfg.weyl_block) if fmt in workloads.SCALED_FORMATS else 0)
     out = open(args.out, "w") if args.out else None
 
     def emit(line):

@@ -6,8 +6,10 @@ import torch
 import oracle
 from paper_2609_39185_b200 import ssdq, workloads
 
-TORCH_CODE = {ssdq.FP16: torch.int16, ssdq.BF16: torch.int16, ssdq.E4M3: torch.uint8, ssdq.FP32: torch.int32}
-NP_VIEW = {ssdq.FP16: np.int16, ssdq.BF16: np.int16, ssdq.E4M3: np.uint8, ssdq.FP32: np.int32}
+TORCH_CODE = {ssdq.FP16: torch.int16, ssdq.BF16: torch.int16, ssdq.E4M3: torch.uint8, ssdq.FP32: torch.int32,
+              ssdq.INT8: torch.uint8, ssdq.INT7: torch.uint8, ssdq.INT6: torch.uint8, ssdq.INT4: torch.uint8}
+NP_VIEW = {ssdq.FP16: np.int16, ssdq.BF16: np.int16, ssdq.E4M3: np.uint8, ssdq.FP32: np.int32,
+           ssdq.INT8: np.uint8, ssdq.INT7: np.uint8, ssdq.INT6: np.uint8, ssdq.INT4: np.uint8}
 
 
 def to_dev(a):

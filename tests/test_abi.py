@@ -65,7 +65,7 @@ def _desc(**over):
     (dict(state=0x10008), ssdq.ERR_ALIGN),
     (dict(Bm=0x10004), ssdq.ERR_ALIGN),
     (dict(dstate=48), ssdq.ERR_UNSUPPORTED),
-    (dict(format=7), ssdq.ERR_UNSUPPORTED),
+    (dict(format=9), ssdq.ERR_UNSUPPORTED),
     (dict(rule=5), ssdq.ERR_UNSUPPORTED),
     (dict(batch=0), ssdq.ERR_SHAPE),
     (dict(format=ssdq.E4M3, scales=None, scale_block=128), ssdq.ERR_NULL),

@@ -10,13 +10,13 @@ from parity import to_dev, codes_to_dev
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("fmt", [ssdq.FP16, ssdq.BF16, ssdq.E4M3, ssdq.FP32])
+@pytest.mark.parametrize("fmt", [ssdq.FP16, ssdq.BF16, ssdq.E4M3, ssdq.FP32, ssdq.INT8])
 def test_state_error_matches_definition(fmt):
     rng = np.random.default_rng(fmt)
     B, H, P, N = 3, 5, 6, 128
     twin = rng.standard_normal((B, H, P, N)).astype(np.float32)
     noisy = (twin * (1 + 0.01 * rng.standard_normal(twin.shape))).astype(np.float32)
-    sb = 128 if fmt == ssdq.E4M3 else 0
+    sb = 128 if oracle.has_block_scale(fmt) else 0
     if fmt == ssdq.FP32:
         codes, scales = noisy.view(np.uint32).reshape(-1, N), None
     else:

@@ -13,6 +13,7 @@ from parity import to_dev, codes_to_host, TORCH_CODE
 pytestmark = pytest.mark.gpu
 
 FMTS = [ssdq.FP16, ssdq.BF16, ssdq.E4M3]
+INT_FMTS = [ssdq.INT8, ssdq.INT7, ssdq.INT6, ssdq.INT4]
 RULES = [ssdq.RTN, ssdq.SR, ssdq.WEYL]
 
 
@@ -40,11 +41,11 @@ def value_zoo(rng, n_rows, row_len, fmt):
     """float32 rows that exercise every branch of Eq. 2 on the local grid: all binades of the format
     including its subnormal range and values below it, exact grid points, zeros of both signs,
     values beyond the largest finite number."""
-    lo, hi = {ssdq.FP16: (-50, 17), ssdq.BF16: (-126, 127), ssdq.E4M3: (-40, 10)}[fmt]
+    lo, hi = {ssdq.FP16: (-50, 17), ssdq.BF16: (-126, 127), ssdq.E4M3: (-40, 10)}.get(fmt, (-40, 10))
     n = n_rows * row_len
     e = rng.integers(lo, hi + 1, n)
     m = rng.integers(0, 1 << 23, n).astype(np.uint32)
-    keep = {ssdq.FP16: 10, ssdq.BF16: 7, ssdq.E4M3: 3}[fmt]
+    keep = {ssdq.FP16: 10, ssdq.BF16: 7, ssdq.E4M3: 3}.get(fmt, 6)
     m[::5] &= np.uint32(~((1 << (23 - keep)) - 1) & 0x7FFFFF)      # exact grid points (in the normal range)
     m[1::11] = 0x7FFFFF                                             # just below a binade boundary
     s = rng.integers(0, 2, n).astype(np.uint32)
@@ -56,14 +57,16 @@ def value_zoo(rng, n_rows, row_len, fmt):
     return bits.view(np.float32).reshape(n_rows, row_len)
 
 
-@pytest.mark.parametrize("fmt", FMTS)
+@pytest.mark.parametrize("fmt", FMTS + INT_FMTS)
 @pytest.mark.parametrize("rule", RULES)
 @pytest.mark.parametrize("row_len,weyl_block,scale_block", [(128, 128, 128), (128, 16, 16), (16, 16, 16), (64, 16, 64), (256, 16, 16), (32, 16, 32)])
 def test_quantize_store_matches_oracle(fmt, rule, row_len, weyl_block, scale_block):
     rng = np.random.default_rng(1000 * fmt + 10 * rule + row_len)
     n_rows = 700                                                    # not a multiple of the slots per CTA
     src = value_zoo(rng, n_rows, row_len, fmt)
-    sb = scale_block if fmt == ssdq.E4M3 else 0
+    sb = scale_block if oracle.has_block_scale(fmt) else 0
+    if fmt in INT_FMTS:      # integer grids: mix blocks of ordinary magnitudes with the zoo (whose blocks are dominated by one huge entry)
+        src[::2] = (rng.standard_normal((len(src[::2]), row_len)) * rng.uniform(1e-3, 50, (len(src[::2]), 1))).astype(np.float32)
     base, t, layer, seed = 2**30 + 5, 1234567, 4, 99
     want_codes, want_scales = oracle.quantize_store(src, fmt, rule, t, scale_block=sb, layer=layer, weyl_seed=1,
                                                     weyl_block=weyl_block, sr_seed=seed, row_index_base=base)
@@ -119,11 +122,11 @@ def test_subnormal_decision_boundary(fmt):
         assert np.array_equal(codes_to_host(codes, fmt), want_codes), trial
 
 
-@pytest.mark.parametrize("fmt", FMTS + [ssdq.FP32])
+@pytest.mark.parametrize("fmt", FMTS + [ssdq.FP32, ssdq.INT8, ssdq.INT4])
 def test_dequantize_matches_oracle(fmt):
     rng = np.random.default_rng(3)
     n_rows, row_len = 33, 128
-    sb = 128 if fmt == ssdq.E4M3 else 0
+    sb = 128 if oracle.has_block_scale(fmt) else 0
     if fmt == ssdq.FP32:
         codes_h = rng.standard_normal((n_rows, row_len)).astype(np.float32).view(np.uint32)
         scales_h = None

@@ -84,6 +84,24 @@ def test_config5_full_batch_launch_sampled_sequences(rule):
         torch.cuda.empty_cache()
 
 
+@pytest.mark.parametrize("rule", RULES)
+@pytest.mark.parametrize("fmt", [ssdq.INT8, ssdq.INT4])
+def test_int_store_on_the_hybrid_shape(rule, fmt):
+    """The paper's headline format (INT8, FP32 block scale, block = state dimension for the hybrids) on the
+    config 4 shape: full size for a few steps, then a long horizon on one sequence."""
+    from dataclasses import replace
+    cfg = replace(CFG[4], fmt=fmt)
+    run_parity(cfg, rule, 3)
+    run_parity(cfg, rule, 512, batch_slice=slice(5, 6), batch_index_base=5, check_every=64)
+
+
+@pytest.mark.parametrize("rule", RULES)
+def test_int8_store_on_the_mamba1_shape(rule):
+    from dataclasses import replace
+    cfg = replace(CFG[2], fmt=ssdq.INT8, scale_block=16)      # blocks of 16 entries for the Mamba models
+    run_parity(cfg, rule, 64, check_every=8)
+
+
 SHAPES = [
     # (B, H, P, N, a_per_state)
     (1, 1, 1, 16, False), (3, 5, 7, 16, True), (2, 3, 64, 128, False), (5, 7, 3, 128, False), (2, 2, 100, 64, False),
@@ -91,7 +109,7 @@ SHAPES = [
 ]
 
 
-@pytest.mark.parametrize("fmt", [ssdq.FP16, ssdq.BF16, ssdq.E4M3, ssdq.FP32])
+@pytest.mark.parametrize("fmt", [ssdq.FP16, ssdq.BF16, ssdq.E4M3, ssdq.FP32, ssdq.INT8, ssdq.INT4])
 @pytest.mark.parametrize("rule", RULES)
 @pytest.mark.parametrize("shape", SHAPES)
 def test_edge_shapes_and_options(fmt, rule, shape):
@@ -105,7 +123,7 @@ def test_edge_shapes_and_options(fmt, rule, shape):
     D = rng.normal(0, 0.1, H).astype(f32) if use_D else None
     wb = 16 if (P + N) % 3 else N
     sb = 0
-    if fmt == ssdq.E4M3:
+    if oracle.has_block_scale(fmt):
         sb = 16 if P % 2 else N
     src = (rng.standard_normal((B * H * P, N)) * 0.3).astype(f32)
     base = 11
@@ -125,14 +143,14 @@ def test_edge_shapes_and_options(fmt, rule, shape):
         pair.compare(t, x, dt, Bm, Cm, y_ref)
 
 
-@pytest.mark.parametrize("fmt", [ssdq.FP16, ssdq.BF16, ssdq.E4M3])
+@pytest.mark.parametrize("fmt", [ssdq.FP16, ssdq.BF16, ssdq.E4M3, ssdq.INT8])
 def test_extreme_values_saturate_and_keep_signed_zero(fmt):
     """Decay to (sub)normal dust, growth beyond the largest finite value, exact zeros of both signs."""
     rng = np.random.default_rng(5)
     B, H, P, N = 1, 4, 4, 128
     f32 = np.float32
     A = np.array([-40.0, -1e-6, -3.0, 0.0], f32)           # fast decay / almost none / medium / a = 1
-    sb = N if fmt == ssdq.E4M3 else 0
+    sb = N if oracle.has_block_scale(fmt) else 0
     for rule in RULES:
         pair = Pair((B, H, P, N), fmt, rule, A, None, weyl_block=N, scale_block=sb)
         for t in range(1, 40):
