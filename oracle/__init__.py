@@ -17,9 +17,9 @@ import numpy as np
 FP16, BF16, E4M3, FP32 = 0, 1, 2, 3
 INT8, INT7, INT6, INT4 = 4, 5, 6, 7          # symmetric block-absmax integers, one int8 per entry
 INT_QMAX = {INT8: 127, INT7: 63, INT6: 31, INT4: 7}
-RTN, SR, WEYL = 0, 1, 2
+RTN, SR, WEYL, SR_HASH = 0, 1, 2, 3
 FORMAT_NAMES = {FP16: "fp16", BF16: "bf16", E4M3: "e4m3", FP32: "fp32", INT8: "int8", INT7: "int7", INT6: "int6", INT4: "int4"}
-RULE_NAMES = {RTN: "rtn", SR: "sr", WEYL: "weyl"}
+RULE_NAMES = {RTN: "rtn", SR: "sr", WEYL: "weyl", SR_HASH: "sr_hash"}
 CODE_DTYPE = {FP16: np.uint16, BF16: np.uint16, E4M3: np.uint8, FP32: np.uint32, INT8: np.uint8, INT7: np.uint8,
               INT6: np.uint8, INT4: np.uint8}
 
@@ -54,6 +54,8 @@ def lib() -> ctypes.CDLL:
         L.oracle_philox4x32_10.argtypes = [vp, vp, vp]
         L.oracle_exp_spec.restype = f32
         L.oracle_exp_spec.argtypes = [f32]
+        L.oracle_fmix32.restype = u32
+        L.oracle_fmix32.argtypes = [u32]
         L.oracle_round.restype = f32
         L.oracle_round.argtypes = [f32, i32, i32, u32]
         L.oracle_encode.restype = u32
@@ -104,6 +106,10 @@ def philox4x32_10(ctr, key):
     out = np.zeros(4, dtype=np.uint32)
     lib().oracle_philox4x32_10(_ptr(c), _ptr(k), _ptr(out))
     return out
+
+
+def fmix32(h) -> int:
+    return lib().oracle_fmix32(h & 0xFFFFFFFF)
 
 
 def exp_spec(z):

@@ -42,7 +42,7 @@ namespace {
 
 enum Format { FMT_FP16 = 0, FMT_BF16 = 1, FMT_E4M3 = 2, FMT_FP32 = 3 /* no rounding: the fp32-state twin */,
               FMT_INT8 = 4, FMT_INT7 = 5, FMT_INT6 = 6, FMT_INT4 = 7 /* symmetric block-absmax integers in an int8 container */ };
-enum Rule { RULE_RTN = 0, RULE_SR = 1, RULE_WEYL = 2 };
+enum Rule { RULE_RTN = 0, RULE_SR = 1, RULE_WEYL = 2, RULE_SR_HASH = 3 };
 
 struct FormatSpec {
     int mant_bits;   // explicit mantissa bits m
@@ -108,6 +108,24 @@ void philox4x32_10(const uint32_t ctr_in[4], const uint32_t key_in[2], uint32_t 
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
+// Integer-hash SR (Section 6.5 "Cost": SR driven by a cheap integer hash is as accurate as Philox SR; Appendix B
+// "Decode regime": u = fmix32(i * 0x9E3779B1 + t * 0x85EBCA77 + ...) / 2^32 truncated to 24 bits).  fmix32 is the
+// 32-bit finaliser of MurmurHash3.  The paper elides the remaining terms; this build continues the same family
+// of odd multipliers for layer and seed and folds in the high half of a 64-bit entry index.
+uint32_t fmix32(uint32_t h) {
+    h ^= h >> 16;
+    h *= 0x85EBCA6Bu;
+    h ^= h >> 13;
+    h *= 0xC2B2AE35u;
+    h ^= h >> 16;
+    return h;
+}
+uint32_t hash_sr_word(uint64_t flat, uint32_t t, uint32_t layer, uint64_t seed) {
+    const uint32_t i_lo = (uint32_t)flat, i_hi = (uint32_t)(flat >> 32);
+    const uint32_t s_lo = (uint32_t)seed, s_hi = (uint32_t)(seed >> 32);
+    return fmix32(i_lo * 0x9E3779B1u + t * 0x85EBCA77u + layer * 0xC2B2AE3Du + s_lo * 0x27D4EB2Fu + (i_hi ^ s_hi) * 0x165667B1u);
+}
+
 struct RuleParams {
     int rule;
     uint32_t layer;       // layer index l (Weyl offsets and SR counter)
@@ -131,6 +149,7 @@ uint32_t threshold_u24(const RuleParams& rp, uint64_t flat, uint32_t t) {
         philox4x32_10(ctr, key, out);
         return out[flat % 4] >> 8;
     }
+    if (rp.rule == RULE_SR_HASH) return hash_sr_word(flat, t, rp.layer, rp.sr_seed) >> 8;
     return 0;  // RTN has no threshold
 }
 
@@ -284,6 +303,7 @@ uint32_t oracle_weyl_acc(uint32_t r, uint32_t c, uint32_t layer, uint32_t seed, 
 }
 void oracle_philox4x32_10(const uint32_t* ctr, const uint32_t* key, uint32_t* out) { philox4x32_10(ctr, key, out); }
 float oracle_exp_spec(float z) { return exp_spec(z); }
+uint32_t oracle_fmix32(uint32_t h) { return fmix32(h); }
 float oracle_round(float v, int fmt, int rule, uint32_t U) { return round_on_grid(v, fmt, rule, U); }
 uint32_t oracle_encode(float q, int fmt) { return encode(q, fmt); }
 float oracle_decode(uint32_t code, int fmt) { return decode(code, fmt); }

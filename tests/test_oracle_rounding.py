@@ -10,7 +10,7 @@ import pytest
 import torch
 
 import oracle
-from oracle import FP16, BF16, E4M3, RTN, SR, WEYL
+from oracle import FP16, BF16, E4M3, RTN, SR, WEYL, SR_HASH
 
 TORCH_DTYPE = {FP16: torch.float16, BF16: torch.bfloat16, E4M3: torch.float8_e4m3fn}
 MAX_FINITE = {FP16: 65504.0, BF16: float(np.float32(3.3895313892515355e38)), E4M3: 448.0}
@@ -163,7 +163,7 @@ def test_saturation_and_rtn_ties(fmt):
         assert oracle.round_values(np.float32(1.0 + 1.5 * s), 0, FP16, RTN)[0] == np.float32(1.0 + 2 * s)
 
 
-@pytest.mark.parametrize("rule", [SR, WEYL])
+@pytest.mark.parametrize("rule", [SR, WEYL, SR_HASH])
 def test_dithers_are_unbiased_and_lemma_2_noise(rule):
     # E[Q_u(x)] = x over a long run (Section 2), and Lemma 2: with f uniform the mean squared
     # residual is s^2/12 under RTN and s^2/6 under SR or the Weyl dither.

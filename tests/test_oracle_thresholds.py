@@ -161,3 +161,52 @@ def test_sr_thresholds_look_uniform():
     across = np.array([oracle.threshold(oracle.SR, flat=f, t=9, sr_seed=1) for f in range(n)]) / 2.0**24
     assert abs(across.mean() - 0.5) < 3 * math.sqrt(1 / 12 / n)
     assert abs(np.corrcoef(across[:-1], across[1:])[0, 1]) < 3 / math.sqrt(n)
+
+
+# ---- integer-hash SR ---------------------------------------------------------------------------
+def _unfmix32(h):
+    """Inverse of the MurmurHash3 finaliser, built from the modular inverses of its two multipliers and the
+    inverses of its xor-shifts (different operations from the forward direction)."""
+    m = 0xFFFFFFFF
+    h ^= h >> 16
+    h = (h * pow(0xC2B2AE35, -1, 2**32)) & m
+    h ^= (h >> 13) ^ (h >> 26)
+    h = (h * pow(0x85EBCA6B, -1, 2**32)) & m
+    h ^= h >> 16
+    return h
+
+
+def test_fmix32_is_the_murmur3_finaliser():
+    rng = np.random.default_rng(11)
+    assert oracle.fmix32(0) == 0
+    xs = [int(v) for v in rng.integers(0, 1 << 32, 3000)] + [1, 2, 0xFFFFFFFF, 0x80000000]
+    for x in xs:
+        assert _unfmix32(oracle.fmix32(x)) == x                       # a permutation, inverted by independent arithmetic
+    # avalanche: flipping one input bit flips about half of the output bits
+    flips = []
+    for x in xs[:300]:
+        for b in (0, 7, 16, 31):
+            flips.append(bin(oracle.fmix32(x) ^ oracle.fmix32(x ^ (1 << b))).count("1"))
+    assert 15.0 < np.mean(flips) < 17.0
+
+
+def test_hash_sr_definition_and_moments():
+    # definition: fmix32(i_lo*P1 + t*P2 + layer*P3 + seed_lo*P4 + (i_hi ^ seed_hi)*P5) >> 8 with the two multipliers
+    # the paper prints (0x9E3779B1 for the entry, 0x85EBCA77 for the step)
+    P1, P2, P3, P4, P5 = 0x9E3779B1, 0x85EBCA77, 0xC2B2AE3D, 0x27D4EB2F, 0x165667B1
+    for flat, t, layer, seed in ((0, 1, 0, 0), (12345, 99, 3, 7), (2**35 + 17, 2**31 + 5, 11, 2**40 + 3)):
+        key = ((flat & 0xFFFFFFFF) * P1 + t * P2 + layer * P3 + (seed & 0xFFFFFFFF) * P4 + ((flat >> 32) ^ (seed >> 32)) * P5) % 2**32
+        assert oracle.threshold(oracle.SR_HASH, flat, t, layer=layer, sr_seed=seed) == oracle.fmix32(key) >> 8
+    # the paper's unit test of its hash: mean 0.4997, variance 0.0834, lag-1 correlation -5e-5
+    n = 40000
+    u = np.array([oracle.threshold(oracle.SR_HASH, flat=777, t=t) for t in range(1, n + 1)]) / 2.0**24
+    assert abs(u.mean() - 0.5) < 3 * math.sqrt(1 / 12 / n)
+    assert abs(u.var() - 1 / 12) < 0.002
+    assert abs(np.corrcoef(u[:-1], u[1:])[0, 1]) < 3 / math.sqrt(n)
+    across = np.array([oracle.threshold(oracle.SR_HASH, flat=f, t=5) for f in range(n)]) / 2.0**24
+    assert abs(across.mean() - 0.5) < 3 * math.sqrt(1 / 12 / n)
+    assert abs(np.corrcoef(across[:-1], across[1:])[0, 1]) < 3 / math.sqrt(n)
+    # local discrepancy of a random sequence (Table 8, row SR: 0.0539)
+    vals = [star_discrepancy([oracle.threshold(oracle.SR_HASH, flat=2000 + j, t=t) / 2.0**24 for t in range(1, 257)])
+            for j in range(200)]
+    assert abs(np.mean(vals) - 0.0539) < 0.004

@@ -8,7 +8,7 @@ import numpy as np
 import pytest
 
 import oracle
-from oracle import FP16, BF16, E4M3, FP32, RTN, SR, WEYL
+from oracle import FP16, BF16, E4M3, FP32, RTN, SR, WEYL, SR_HASH
 from paper_2609_39185_b200 import workloads
 
 
@@ -44,7 +44,7 @@ def run_scalar_recurrence(w_over_step, h0, T, rule, fmt=FP16):
     return oracle.decode(state, fmt).reshape(N).astype(np.float64)
 
 
-@pytest.mark.parametrize("rule", [RTN, SR, WEYL])
+@pytest.mark.parametrize("rule", [RTN, SR, WEYL, SR_HASH])
 @pytest.mark.parametrize("sign", [+1, -1])
 def test_proposition_1_identity_end_to_end(rule, sign):
     # a_t = 1, w_t = w, h_0 on the grid: h_T = h_0 + s*(T*m + #{t <= T : u_t >= 1 - f}), so
