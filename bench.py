@@ -28,7 +28,7 @@ sys.path.insert(0, ROOT)
 
 from paper_2609_39185_b200 import workloads  # noqa: E402
 
-RULE_IDS = {"rtn": 0, "sr": 1, "weyl": 2}
+RULE_IDS = {"rtn": 0, "sr": 1, "weyl": 2, "sr_hash": 3}
 NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the fused update kernel, from the ncu
 # captures summarised under profiles/ (same kernel and per-layer shape as the benchmark's launches).
@@ -317,7 +317,7 @@ def main():
     if not args.no_extras:
         # ---- per-rule sweep: interleaved rounds over {copy, rtn, sr, weyl}, median per rule ----
         rounds, reps = 7, max(10, min(50, args.steps))
-        times = {k: [] for k in ("copy", "rtn", "sr", "weyl")}
+        times = {k: [] for k in ("copy", "rtn", "sr", "weyl", "sr_hash")}
         dst = torch.empty_like(stack.states[0])
         for _ in range(rounds):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -338,6 +338,7 @@ def main():
                              "gbs": (copy_bytes if k == "copy" else bytes_per_step) / med[k] / 1e9} for k in med}
         line["weyl_over_rtn_time"] = med["weyl"] / med["rtn"]
         line["sr_over_rtn_time"] = med["sr"] / med["rtn"]
+        line["sr_hash_over_rtn_time"] = med["sr_hash"] / med["rtn"]
 
         # ---- end to end: per step, inputs come from pinned host memory and y goes back to the host ----
         in_bytes = sum(t[0].numel() * 4 for t in (xs_h, dts_h, Bs_h, Cs_h))

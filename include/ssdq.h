@@ -49,8 +49,11 @@ typedef enum {
     SSDQ_INT8 = 4, SSDQ_INT7 = 5, SSDQ_INT6 = 6, SSDQ_INT4 = 7
 } ssdq_format;
 
-/* Threshold rules of Eq. 2.  RTN rounds to nearest, ties to even (the rule of native casts). */
-typedef enum { SSDQ_RTN = 0, SSDQ_SR_PHILOX = 1, SSDQ_WEYL = 2 } ssdq_rule;
+/* Threshold rules of Eq. 2.  RTN rounds to nearest, ties to even (the rule of native casts).
+ * SSDQ_SR_HASH is stochastic rounding driven by a cheap integer hash instead of Philox (Section 6.5 "Cost";
+ * Appendix B "Decode regime"): U = fmix32(i_lo*0x9E3779B1 + t*0x85EBCA77 + layer*0xC2B2AE3D + seed_lo*0x27D4EB2F
+ * + (i_hi ^ seed_hi)*0x165667B1) >> 8 with i the flat entry index, seed = sr_seed, fmix32 the MurmurHash3 finaliser. */
+typedef enum { SSDQ_RTN = 0, SSDQ_SR_PHILOX = 1, SSDQ_WEYL = 2, SSDQ_SR_HASH = 3 } ssdq_rule;
 
 /* Weyl dither in 32-bit fixed point (Appendix B "Dithers", hardware form):
  *   acc(r, c, t) = mul_row*(r+1) + mul_col*(c+1) + base + t*phi   (mod 2^32),   u = (acc >> 8) / 2^24
@@ -73,7 +76,7 @@ int weyl_offsets_init(ssdq_weyl* out, uint32_t layer, uint32_t seed, uint32_t bl
 /* Test aid: write the 24-bit thresholds U of entries flat = first_flat .. first_flat + n - 1 at
  * write index step_t into out_u24 (DEVICE, n x uint32).  rule = SSDQ_WEYL uses `weyl`;
  * SSDQ_SR_PHILOX uses Philox4x32-10 with key = sr_seed and counter = (flat/4 low, flat/4 high,
- * step_t, layer), word flat % 4, top 24 bits; SSDQ_RTN writes zeros. */
+ * step_t, layer), word flat % 4, top 24 bits; SSDQ_SR_HASH as defined at ssdq_rule; SSDQ_RTN writes zeros. */
 int ssdq_thresholds_materialize(int rule, const ssdq_weyl* weyl, uint64_t sr_seed, uint32_t layer,
                                 uint64_t first_flat, uint64_t n, uint32_t step_t, uint32_t* out_u24, void* stream);
 

@@ -61,7 +61,7 @@ int check_layer(const ssdq_update_desc* d) {
     if (!d) return fail(SSDQ_ERR_NULL, "descriptor is NULL");
     if (d->batch == 0 || d->nheads == 0 || d->headdim == 0) return fail(SSDQ_ERR_SHAPE, "batch, nheads and headdim must be positive");
     if (!format_known(d->format)) return fail(SSDQ_ERR_UNSUPPORTED, "unknown format %d", d->format);
-    if (d->rule < SSDQ_RTN || d->rule > SSDQ_WEYL) return fail(SSDQ_ERR_UNSUPPORTED, "unknown rule %d", d->rule);
+    if (d->rule < SSDQ_RTN || d->rule > SSDQ_SR_HASH) return fail(SSDQ_ERR_UNSUPPORTED, "unknown rule %d", d->rule);
     if (!dstate_supported(d->format, d->dstate)) return fail(SSDQ_ERR_UNSUPPORTED, "dstate %u is not supported for format %d", d->dstate, d->format);
     if ((uint64_t)d->batch * d->nheads > 0xFFFFFFFFull / 2) return fail(SSDQ_ERR_SHAPE, "batch * nheads too large");
     if (!d->state || !d->A) return fail(SSDQ_ERR_NULL, "state and A are required");
@@ -182,7 +182,7 @@ int weyl_offsets_init(ssdq_weyl* out, uint32_t layer, uint32_t seed, uint32_t bl
 
 int ssdq_thresholds_materialize(int rule, const ssdq_weyl* weyl, uint64_t sr_seed, uint32_t layer, uint64_t first_flat,
                                 uint64_t n, uint32_t step_t, uint32_t* out_u24, void* stream) {
-    if (rule < SSDQ_RTN || rule > SSDQ_WEYL) return fail(SSDQ_ERR_UNSUPPORTED, "unknown rule %d", rule);
+    if (rule < SSDQ_RTN || rule > SSDQ_SR_HASH) return fail(SSDQ_ERR_UNSUPPORTED, "unknown rule %d", rule);
     if (n && !out_u24) return fail(SSDQ_ERR_NULL, "out_u24 is NULL");
     ssdq::WeylConst w{};
     if (rule == SSDQ_WEYL) {
@@ -209,7 +209,7 @@ int quantize_store(const float* src, void* dst_codes, float* dst_scales, uint64_
                    uint32_t scale_block, int format, int rule, const ssdq_weyl* weyl, uint64_t sr_seed, uint32_t layer,
                    uint64_t row_index_base, uint32_t step_t, void* stream) {
     if (!format_known(format)) return fail(SSDQ_ERR_UNSUPPORTED, "unknown format %d", format);
-    if (rule < SSDQ_RTN || rule > SSDQ_WEYL) return fail(SSDQ_ERR_UNSUPPORTED, "unknown rule %d", rule);
+    if (rule < SSDQ_RTN || rule > SSDQ_SR_HASH) return fail(SSDQ_ERR_UNSUPPORTED, "unknown rule %d", rule);
     if (!dstate_supported(format, row_len)) return fail(SSDQ_ERR_UNSUPPORTED, "row_len %u is not supported for format %d", row_len, format);
     if (n_rows == 0) return SSDQ_OK;
     if (!src || !dst_codes) return fail(SSDQ_ERR_NULL, "src and dst_codes are required");

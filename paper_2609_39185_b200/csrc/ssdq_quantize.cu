@@ -49,6 +49,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantParams p)
         const uint64_t grow = p.row_base + row;
         uint32_t g_lo = 0, g_hi = 0, acc0 = 0;
         if constexpr (RULE == RULE_WEYL) acc0 = thr.weyl_acc0(grow);
+        if constexpr (RULE == RULE_SR_HASH) acc0 = thr.hash_key0(grow, p.step_t * kHashP2 + p.layer * kHashP3 + key0 * kHashP4, key1);
         if constexpr (RULE == RULE_SR) thr.sr_group(grow, g_lo, g_hi);
         const uint4 packed = round_pack_lane<FMT, RULE>(v, acc0, p.weyl.mul_col, g_lo, g_hi, p.step_t, p.layer, key0, key1, p.scale_top);
         if (ok) reinterpret_cast<uint4*>(p.codes)[row * LPR + lis] = packed;
@@ -87,6 +88,7 @@ static cudaError_t launch_quantize_fmt(const QuantParams& p, int rule, cudaStrea
         case RULE_RTN: return launch_quantize_n<FMT, RULE_RTN>(p, s);
         case RULE_SR: return launch_quantize_n<FMT, RULE_SR>(p, s);
         case RULE_WEYL: return launch_quantize_n<FMT, RULE_WEYL>(p, s);
+        case RULE_SR_HASH: return launch_quantize_n<FMT, RULE_SR_HASH>(p, s);
         default: return cudaErrorInvalidValue;
     }
 }
@@ -153,6 +155,10 @@ __global__ void __launch_bounds__(256) thresholds_kernel(int rule, WeylConst w, 
                                           (uint32_t)sr_seed, (uint32_t)(sr_seed >> 32));
             const uint32_t word[4] = {o.x, o.y, o.z, o.w};
             U = word[flat & 3u] >> 8;
+        } else if (rule == RULE_SR_HASH) {
+            const uint32_t key = (uint32_t)flat * kHashP1 + step_t * kHashP2 + layer * kHashP3 + (uint32_t)sr_seed * kHashP4 +
+                                 ((uint32_t)(flat >> 32) ^ (uint32_t)(sr_seed >> 32)) * kHashP5;
+            U = fmix32(key) >> 8;
         }
         out[i] = U;
     }

@@ -77,6 +77,9 @@ __device__ __forceinline__ uint4 round_pack_lane(const float* v, uint32_t acc0, 
         if constexpr (RULE == RULE_WEYL) {
 #pragma unroll
             for (int k = 0; k < EPL; ++k) acc[k] = acc0 + (uint32_t)k * mul_col;
+        } else if constexpr (RULE == RULE_SR_HASH) {
+#pragma unroll
+            for (int k = 0; k < EPL; ++k) acc[k] = fmix32(acc0 + (uint32_t)k * kHashP1);    // acc0 = hash key of the first entry
         } else {
 #pragma unroll
             for (int g = 0; g < EPL / 4; ++g) {
@@ -157,6 +160,11 @@ struct LaneThreshold {
         }
     }
     __device__ __forceinline__ uint32_t weyl_acc0(uint64_t grow) const { return lane_const + row_mul * (uint32_t)grow; }
+    // hash SR: key of the lane's first entry in row `grow`; hash_base = t*P2 + layer*P3 + seed_lo*P4
+    __device__ __forceinline__ uint32_t hash_key0(uint64_t grow, uint32_t hash_base, uint32_t seed_hi) const {
+        const uint64_t flat = grow * (uint64_t)N + n0;
+        return (uint32_t)flat * kHashP1 + ((uint32_t)(flat >> 32) ^ seed_hi) * kHashP5 + hash_base;
+    }
     __device__ __forceinline__ void sr_group(uint64_t grow, uint32_t& g_lo, uint32_t& g_hi) const {
         const uint64_t g = (grow * (uint64_t)N + n0) >> 2;
         g_lo = (uint32_t)g;
@@ -215,6 +223,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_kernel(const UpdateParams
     thr.init(p.weyl, p.step_t, lis);
     const uint32_t key0 = (uint32_t)p.sr_seed, key1 = (uint32_t)(p.sr_seed >> 32);
 
+    const uint32_t hash_base = p.step_t * kHashP2 + p.layer * kHashP3 + key0 * kHashP4;
     const uint32_t p_first = sub * p.rps;                         // first row of this slot inside the item
     const uint64_t row_first = (uint64_t)item * p.P + p_first;    // local row index (this call's tensors)
     const uint64_t grow_first = row_first + (uint64_t)p.batch_base * p.H * p.P;   // global row index
@@ -280,6 +289,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_kernel(const UpdateParams
             }
             uint32_t g_lo = 0, g_hi = 0, acc0 = 0;
             if constexpr (RULE == RULE_WEYL) acc0 = thr.weyl_acc0(grow_first + k);
+            if constexpr (RULE == RULE_SR_HASH) acc0 = thr.hash_key0(grow_first + k, hash_base, key1);
             if constexpr (RULE == RULE_SR) thr.sr_group(grow_first + k, g_lo, g_hi);
             const uint4 packed = round_pack_lane<FMT, RULE>(hv, acc0, p.weyl.mul_col, g_lo, g_hi, p.step_t, p.layer,
                                                              key0, key1, p.scale_top);
@@ -376,6 +386,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
     const uint64_t grow_first = row_first + (uint64_t)p.batch_base * p.H * (NSLOT * RPS);
     uint32_t acc_row = 0;
     uint64_t grp_row = 0;
+    const uint32_t hash_base = p.step_t * kHashP2 + p.layer * kHashP3 + key0 * kHashP4;
     if constexpr (RULE == RULE_WEYL) acc_row = thr.weyl_acc0(grow_first);
     if constexpr (RULE == RULE_SR) grp_row = (grow_first * (uint64_t)N + n0) >> 2;
 
@@ -412,6 +423,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
                 if (row_scale) { if (lis == 0) p.scales[row_first + k] = s; }
                 else p.scales[(row_first + k) * (N / 16) + lis] = s;
             }
+            if constexpr (RULE == RULE_SR_HASH) acc_row = thr.hash_key0(grow_first + k, hash_base, key1);
             const uint4 packed = round_pack_lane<FMT, RULE>(hv, acc_row, p.weyl.mul_col, (uint32_t)grp_row,
                                                              (uint32_t)(grp_row >> 32), p.step_t, p.layer, key0, key1, p.scale_top);
             sp[k * LPR] = packed;
@@ -476,6 +488,7 @@ inline cudaError_t launch_update_fmt(const UpdateParams& p, int rule, bool aps, 
             case RULE_RTN: return aps ? launch_update_n<FMT, RULE_RTN, true>(p, stream) : launch_update_n<FMT, RULE_RTN, false>(p, stream);
             case RULE_SR: return aps ? launch_update_n<FMT, RULE_SR, true>(p, stream) : launch_update_n<FMT, RULE_SR, false>(p, stream);
             case RULE_WEYL: return aps ? launch_update_n<FMT, RULE_WEYL, true>(p, stream) : launch_update_n<FMT, RULE_WEYL, false>(p, stream);
+            case RULE_SR_HASH: return aps ? launch_update_n<FMT, RULE_SR_HASH, true>(p, stream) : launch_update_n<FMT, RULE_SR_HASH, false>(p, stream);
             default: return cudaErrorInvalidValue;
         }
     }

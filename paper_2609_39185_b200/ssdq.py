@@ -11,7 +11,7 @@ import os
 
 FP16, BF16, E4M3, FP32 = 0, 1, 2, 3
 INT8, INT7, INT6, INT4 = 4, 5, 6, 7
-RTN, SR, WEYL = 0, 1, 2
+RTN, SR, WEYL, SR_HASH = 0, 1, 2, 3
 OK, ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_UNSUPPORTED, ERR_CUDA = 0, -1, -2, -3, -4, -5
 
 _HERE = os.path.dirname(os.path.abspath(__file__))

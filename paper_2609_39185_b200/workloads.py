@@ -18,9 +18,9 @@ import numpy as np
 FP16, BF16, E4M3, FP32 = 0, 1, 2, 3
 INT8, INT7, INT6, INT4 = 4, 5, 6, 7
 SCALED_FORMATS = (E4M3, INT8, INT7, INT6, INT4)
-RTN, SR, WEYL = 0, 1, 2
+RTN, SR, WEYL, SR_HASH = 0, 1, 2, 3
 FORMAT_NAMES = {FP16: "fp16", BF16: "bf16", E4M3: "e4m3", FP32: "fp32", INT8: "int8", INT7: "int7", INT6: "int6", INT4: "int4"}
-RULE_NAMES = {RTN: "rtn", SR: "sr", WEYL: "weyl"}
+RULE_NAMES = {RTN: "rtn", SR: "sr", WEYL: "weyl", SR_HASH: "sr_hash"}
 CODE_BYTES = {FP16: 2, BF16: 2, E4M3: 1, FP32: 4, INT8: 1, INT7: 1, INT6: 1, INT4: 1}
 
 _T_A, _T_D, _T_X, _T_DT, _T_B, _T_C, _T_H0 = range(7)

@@ -66,7 +66,7 @@ def _desc(**over):
     (dict(Bm=0x10004), ssdq.ERR_ALIGN),
     (dict(dstate=48), ssdq.ERR_UNSUPPORTED),
     (dict(format=9), ssdq.ERR_UNSUPPORTED),
-    (dict(rule=5), ssdq.ERR_UNSUPPORTED),
+    (dict(rule=7), ssdq.ERR_UNSUPPORTED),
     (dict(batch=0), ssdq.ERR_SHAPE),
     (dict(format=ssdq.E4M3, scales=None, scale_block=128), ssdq.ERR_NULL),
     (dict(format=ssdq.E4M3, scales=0x20000, scale_block=64), ssdq.ERR_SHAPE),

@@ -14,7 +14,7 @@ pytestmark = pytest.mark.gpu
 
 FMTS = [ssdq.FP16, ssdq.BF16, ssdq.E4M3]
 INT_FMTS = [ssdq.INT8, ssdq.INT7, ssdq.INT6, ssdq.INT4]
-RULES = [ssdq.RTN, ssdq.SR, ssdq.WEYL]
+RULES = [ssdq.RTN, ssdq.SR, ssdq.WEYL, ssdq.SR_HASH]
 
 
 @pytest.mark.parametrize("first_flat", [0, 12345, 2**32 - 100, 2**36 + 3])
@@ -28,12 +28,13 @@ def test_weyl_thresholds_match_oracle(first_flat, block):
         assert np.array_equal(got, want)
 
 
-@pytest.mark.parametrize("first_flat", [0, 7, 2**34 + 1])
-def test_philox_thresholds_match_oracle(first_flat):
+@pytest.mark.parametrize("first_flat", [0, 7, 2**34 + 1, 2**32 - 50])
+@pytest.mark.parametrize("rule", [ssdq.SR, ssdq.SR_HASH])
+def test_sr_thresholds_match_oracle(first_flat, rule):
     n = 4099
     for layer, seed, t in ((0, 0, 1), (3, 0xDEADBEEFCAFE, 77)):
-        got = ssdq.thresholds_materialize(ssdq.SR, n, t, sr_seed=seed, layer=layer, first_flat=first_flat).cpu().numpy().view(np.uint32)
-        want = oracle.thresholds(oracle.SR, range(first_flat, first_flat + n), t, layer=layer, sr_seed=seed)
+        got = ssdq.thresholds_materialize(rule, n, t, sr_seed=seed, layer=layer, first_flat=first_flat).cpu().numpy().view(np.uint32)
+        want = oracle.thresholds(rule, range(first_flat, first_flat + n), t, layer=layer, sr_seed=seed)
         assert np.array_equal(got, want)
 
 

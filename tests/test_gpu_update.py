@@ -10,7 +10,7 @@ from parity import Pair, run_parity, to_dev, codes_to_dev, codes_to_host
 
 pytestmark = pytest.mark.gpu
 
-RULES = [ssdq.RTN, ssdq.SR, ssdq.WEYL]
+RULES = [ssdq.RTN, ssdq.SR, ssdq.WEYL, ssdq.SR_HASH]
 CFG = workloads.CONFIGS
 
 
