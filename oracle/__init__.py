@@ -70,7 +70,9 @@ def lib() -> ctypes.CDLL:
         L.oracle_exp_spec_array.argtypes = [vp, u64, vp]
         L.oracle_state_update.restype = i32
         L.oracle_state_update.argtypes = [vp, vp, i32, u32, u32, u32, u32, u32, vp, vp, vp, i32, vp, vp, vp, vp,
-                                          i32, u32, u32, u32, u64, u32, u32]
+                                          i32, u32, u32, u32, u64, u32, u32, vp, i32, u32, vp]
+        L.oracle_softplus_spec.restype = f32
+        L.oracle_softplus_spec.argtypes = [f32]
         L.oracle_quantize_store.restype = i32
         L.oracle_quantize_store.argtypes = [vp, vp, vp, u64, u32, i32, u32, i32, u32, u32, u32, u64, u64, u32]
         L.oracle_dequantize.restype = None
@@ -150,18 +152,28 @@ def decode(codes, fmt):
 
 
 # ---- the decode step ------------------------------------------------------------------------
+def softplus_spec(x):
+    x = _f32(np.atleast_1d(x))
+    return np.array([lib().oracle_softplus_spec(float(v)) for v in x.ravel()], dtype=np.float32).reshape(x.shape)
+
+
 def state_update(state, scales, fmt, scale_block, x, dt, A, Bm, Cm, D, rule, step_t, *, layer=0,
-                 weyl_seed=0, weyl_block=16, sr_seed=0, batch_index_base=0):
+                 weyl_seed=0, weyl_block=16, sr_seed=0, batch_index_base=0, dt_bias=None, dt_softplus=False,
+                 ngroups=1, z=None):
     """One decode step of one layer, in place on `state` (and `scales`).  Returns y [B,H,P] float32.
 
     state [B,H,P,N] of CODE_DTYPE[fmt] (float32 viewed as uint32 for FP32); x [B,H,P]; dt [B,H];
-    A [H] or [H,N]; Bm, Cm [B,N]; D [H] or None.
+    A [H] or [H,N]; Bm, Cm [B,N] (or [B,G,N] with ngroups=G); D [H] or None; dt_bias [H] or None; with
+    dt_softplus the step size is softplus_spec(dt + dt_bias); z [B,H,P] or None gates y by z * sigmoid(z).
     """
     Bsz, H, P, N = state.shape
     assert state.flags.c_contiguous and state.dtype == CODE_DTYPE[fmt]
     x, dt, A, Bm, Cm = _f32(x), _f32(dt), _f32(A), _f32(Bm), _f32(Cm)
     D = None if D is None else _f32(D)
-    assert x.shape == (Bsz, H, P) and dt.shape == (Bsz, H) and Bm.shape == (Bsz, N) and Cm.shape == (Bsz, N)
+    gshape = (Bsz, N) if ngroups == 1 else (Bsz, ngroups, N)
+    assert x.shape == (Bsz, H, P) and dt.shape == (Bsz, H) and Bm.shape == gshape and Cm.shape == gshape
+    dt_bias = None if dt_bias is None else _f32(dt_bias)
+    z = None if z is None else _f32(z)
     a_per_state = int(A.ndim == 2)
     assert A.shape == ((H, N) if a_per_state else (H,))
     y = np.empty((Bsz, H, P), dtype=np.float32)
@@ -169,7 +181,8 @@ def state_update(state, scales, fmt, scale_block, x, dt, A, Bm, Cm, D, rule, ste
         assert scales.dtype == np.float32 and scales.flags.c_contiguous
     rc = lib().oracle_state_update(_ptr(state), _ptr(scales), fmt, scale_block, Bsz, H, P, N, _ptr(x), _ptr(dt),
                                    _ptr(A), a_per_state, _ptr(Bm), _ptr(Cm), _ptr(D), _ptr(y), rule, layer,
-                                   weyl_seed, weyl_block, sr_seed, batch_index_base, step_t)
+                                   weyl_seed, weyl_block, sr_seed, batch_index_base, step_t, _ptr(dt_bias),
+                                   int(bool(dt_softplus)), ngroups, _ptr(z))
     if rc != 0:
         raise ValueError("oracle_state_update: undefined argument combination")
     return y

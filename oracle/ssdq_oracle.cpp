@@ -285,6 +285,26 @@ float exp_spec(float z) {
     return std::ldexp(p, (int)k);  // exact: the result is a normal number for z in [-87, 88]
 }
 
+// softplus_spec: dt = softplus(dt_raw + dt_bias) feeds the decay and the write term, so like exp_spec it has to be
+// one fixed sequence of binary32 operations.  softplus(x) = max(x, 0) + log1p(exp(-|x|)), and for t in (0, 1]
+// log1p(t) = 2 atanh(u) with u = t / (2 + t) <= 1/3: an odd series in u, cut after u^15 (relative 1e-9).  Above
+// 20 the function returns x, the customary threshold of selective-state-update implementations.
+float softplus_spec(float x) {
+    if (x > 20.0f) return x;
+    const float t = exp_spec(-std::fabs(x));
+    const float u = t / (2.0f + t);
+    const float s = u * u;
+    float p = 0x1.111112p-3f;            // 2/15
+    p = std::fmaf(p, s, 0x1.3b13b2p-3f); // 2/13
+    p = std::fmaf(p, s, 0x1.745d18p-3f); // 2/11
+    p = std::fmaf(p, s, 0x1.c71c72p-3f); // 2/9
+    p = std::fmaf(p, s, 0x1.24924ap-2f); // 2/7
+    p = std::fmaf(p, s, 0x1.99999ap-2f); // 2/5
+    p = std::fmaf(p, s, 0x1.555556p-1f); // 2/3
+    p = std::fmaf(p, s, 2.0f);
+    return std::fmaf(u, p, std::max(x, 0.0f));
+}
+
 // Block scale of the E4M3 store: s = max|h'| / 448 in FP32 (Appendix B "Formats"), floored at the
 // smallest normal number so that an all-zero block is well defined.  Entries are multiplied by
 // 1/s, rounded once per block, instead of being divided by s one by one.
@@ -304,6 +324,7 @@ uint32_t oracle_weyl_acc(uint32_t r, uint32_t c, uint32_t layer, uint32_t seed, 
 void oracle_philox4x32_10(const uint32_t* ctr, const uint32_t* key, uint32_t* out) { philox4x32_10(ctr, key, out); }
 float oracle_exp_spec(float z) { return exp_spec(z); }
 uint32_t oracle_fmix32(uint32_t h) { return fmix32(h); }
+float oracle_softplus_spec(float x) { return softplus_spec(x); }
 float oracle_round(float v, int fmt, int rule, uint32_t U) { return round_on_grid(v, fmt, rule, U); }
 uint32_t oracle_encode(float q, int fmt) { return encode(q, fmt); }
 float oracle_decode(uint32_t code, int fmt) { return decode(code, fmt); }
@@ -322,14 +343,21 @@ void oracle_exp_spec_array(const float* z, uint64_t n, float* out) {
 // ---- one decode step of one layer (Eq. 1 + readout + Eq. 2), in place -----------------------
 // state  : [B, H, P, N] codes of `fmt` (FMT_FP32: floats, no rounding = the fp32-state twin)
 // scales : E4M3 only, [B, H, P, N / scale_block] floats, or [B, H] when scale_block == P * N
-// x [B,H,P], dt [B,H], A [H] or [H,N] (a_per_state), Bm, Cm [B,N], D [H] or null, y [B,H,P]
+// x [B,H,P], dt [B,H], A [H] or [H,N] (a_per_state), Bm, Cm [B,G,N], D [H] or null, y [B,H,P]
+// The rest of a production selective-state-update signature (Appendix B "Runners": grouped B and C, gating as in
+// the reference implementations): dt_bias [H] or null, dt_softplus (dt <- softplus_spec(dt + dt_bias)), ngroups G
+// (head h reads group h / (H / G)), z [B,H,P] or null (y <- y * z * sigmoid(z)).
 // Returns 0, or -1 on an argument the oracle does not define.
 int oracle_state_update(void* state, float* scales, int fmt, uint32_t scale_block,
                         uint32_t B, uint32_t H, uint32_t P, uint32_t N,
                         const float* x, const float* dt, const float* A, int a_per_state,
                         const float* Bm, const float* Cm, const float* D, float* y,
                         int rule, uint32_t layer, uint32_t weyl_seed, uint32_t weyl_block, uint64_t sr_seed,
-                        uint32_t batch_index_base, uint32_t step_t) {
+                        uint32_t batch_index_base, uint32_t step_t,
+                        const float* dt_bias, int dt_softplus, uint32_t ngroups, const float* z) {
+    if (ngroups == 0) ngroups = 1;
+    if (H % ngroups != 0) return -1;
+    const uint32_t heads_per_group = H / ngroups;
     if (has_block_scale(fmt)) {
         if (scale_block == 0 || !scales) return -1;
         if (!(scale_block == P * N || N % scale_block == 0)) return -1;
@@ -341,7 +369,11 @@ int oracle_state_update(void* state, float* scales, int fmt, uint32_t scale_bloc
 #pragma omp parallel for schedule(static)
     for (int64_t bh = 0; bh < BH; ++bh) {
         const uint32_t b = (uint32_t)(bh / H), h = (uint32_t)(bh % H);
-        const float dtv = dt[bh];
+        float dtv = dt[bh];
+        if (dt_bias) dtv = dtv + dt_bias[h];
+        if (dt_softplus) dtv = softplus_spec(dtv);
+        const float* Bg = Bm + ((uint64_t)b * ngroups + h / heads_per_group) * N;
+        const float* Cg = Cm + ((uint64_t)b * ngroups + h / heads_per_group) * N;
         std::vector<float> hp((size_t)P * N);
         // Eq. 1 in FP32: a = exp(dt*A), w = (dt*x)*B, h' = fma(a, h, w); dequantise first.
         for (uint32_t p = 0; p < P; ++p) {
@@ -356,13 +388,17 @@ int oracle_state_update(void* state, float* scales, int fmt, uint32_t scale_bloc
                 }
                 const float Av = a_per_state ? A[(uint64_t)h * N + n] : A[h];
                 const float a = exp_spec(dtv * Av);
-                const float w = dtx * Bm[(uint64_t)b * N + n];
+                const float w = dtx * Bg[n];
                 hp[(size_t)p * N + n] = std::fmaf(a, hv, w);
             }
             // readout from the unrounded h', accumulated in double and rounded once
             double acc = 0.0;
-            for (uint32_t n = 0; n < N; ++n) acc += (double)Cm[(uint64_t)b * N + n] * (double)hp[(size_t)p * N + n];
+            for (uint32_t n = 0; n < N; ++n) acc += (double)Cg[n] * (double)hp[(size_t)p * N + n];
             if (D) acc += (double)D[h] * (double)xv;
+            if (z) {
+                const double zv = (double)z[(uint64_t)bh * P + p];
+                acc *= zv / (1.0 + std::exp(-zv));
+            }
             y[(uint64_t)bh * P + p] = (float)acc;
         }
         // write-back: block scale (E4M3), threshold, Eq. 2, encode

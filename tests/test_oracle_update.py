@@ -245,3 +245,49 @@ def test_sharding_invariance_of_indices():
             y2 = oracle.state_update(part, None, FP16, 0, x[2:], dt[2:], A, Bm[2:], Cm[2:], D, rule, t,
                                      batch_index_base=2)
             assert np.array_equal(full[2:], part) and np.array_equal(y[2:], y2)
+
+
+# ---- the rest of a production signature: dt_bias + softplus, grouped B/C, z gate -----------------
+def test_softplus_spec_accuracy():
+    rng = np.random.default_rng(6)
+    x = np.concatenate([rng.uniform(-100, 25, 200000), rng.uniform(-2, 2, 50000), [0.0, -0.0, 20.0, 20.000002, -87.0, -200.0]]).astype(np.float32)
+    got = oracle.softplus_spec(x).astype(np.float64)
+    xd = x.astype(np.float64)
+    want = np.where(xd > 20.0, xd, np.maximum(xd, 0.0) + np.log1p(np.exp(-np.abs(np.maximum(xd, -87.0)))))
+    ulp = np.spacing(want.astype(np.float32)).astype(np.float64)
+    assert np.max(np.abs(got - want) / ulp) <= 3.0
+    assert np.all(got > 0.0)
+    xs = np.sort(x)
+    assert np.all(np.diff(oracle.softplus_spec(xs).astype(np.float64)) >= -2 * np.spacing(oracle.softplus_spec(xs))[1:])
+
+
+def test_full_signature_reduces_to_the_plain_step():
+    """dt_bias + softplus, grouped B/C and the z gate, each checked against the plain step on transformed inputs:
+    softplus outside the call; per-head copies of the group's B and C; y multiplied by silu(z) afterwards."""
+    rng = np.random.default_rng(8)
+    Bsz, H, P, N, G = 2, 6, 4, 32, 3
+    f32 = np.float32
+    A = -np.exp(rng.uniform(-3, 1, H)).astype(f32)
+    D = rng.normal(0, 0.1, H).astype(f32)
+    bias = rng.normal(-1, 0.5, H).astype(f32)
+    for rule in (RTN, WEYL, SR_HASH):
+        st_a = np.zeros((Bsz, H, P, N), np.uint16)
+        st_b = [np.zeros((Bsz, 1, P, N), np.uint16) for _ in range(H)]
+        for t in range(1, 6):
+            x = rng.standard_normal((Bsz, H, P)).astype(f32)
+            raw = rng.normal(-1, 1, (Bsz, H)).astype(f32)
+            Bm = rng.standard_normal((Bsz, G, N)).astype(f32)
+            Cm = rng.standard_normal((Bsz, G, N)).astype(f32)
+            z = rng.standard_normal((Bsz, H, P)).astype(f32)
+            y = oracle.state_update(st_a, None, BF16, 0, x, raw, A, Bm, Cm, D, rule, t, weyl_block=16, dt_bias=bias,
+                                    dt_softplus=True, ngroups=G, z=z)
+            dt = oracle.softplus_spec((raw + bias[None, :]).astype(f32))
+            for h in range(H):          # one head at a time with its group's B, C; indices differ, so only RTN state is comparable
+                g = h // (H // G)
+                yh = oracle.state_update(st_b[h], None, BF16, 0, x[:, h:h + 1], dt[:, h:h + 1], A[h:h + 1], Bm[:, g], Cm[:, g],
+                                         D[h:h + 1], RTN, t)
+                if rule == RTN:
+                    assert np.array_equal(st_a[:, h:h + 1], st_b[h])
+                    zz = z[:, h:h + 1].astype(np.float64)
+                    want = yh.astype(np.float64) * zz / (1 + np.exp(-zz))
+                    assert np.allclose(y[:, h:h + 1], want, rtol=2e-6, atol=1e-7)
