@@ -101,12 +101,19 @@ typedef struct {
     uint64_t sr_seed;    /* Philox key when rule == SSDQ_SR_PHILOX */
     uint32_t layer;      /* layer index in the SR counter (the Weyl layer term sits in weyl.base) */
     uint32_t batch_index_base;  /* global index of local sequence 0 */
+    /* The rest of a production selective-state-update signature (Appendix B "Runners": grouped B and C, gating as
+     * in the reference implementations).  All optional: zero / NULL gives the plain step. */
+    const float* dt_bias;/* [H] or NULL: added to dt (one rounded add) */
+    const float* z;      /* [B, H, P] or NULL: y <- y * z * sigmoid(z) */
+    uint32_t dt_softplus;/* 1: dt <- softplus_spec(dt + dt_bias), the library's fixed binary32 softplus */
+    uint32_t ngroups;    /* G > 1: Bm, Cm are [B, G, N] and head h reads group h / (H / G); 0 or 1: one group */
 } ssdq_update_desc;
 
 /* One fused decode step of one layer (Eq. 1, readout, Eq. 2), in place, one kernel launch:
  *   h  = dequant(state)                          (E4M3: code * scale, one rounded multiply)
+ *   dt = softplus_spec(dt + dt_bias) if dt_softplus (else dt + dt_bias, else dt)
  *   a  = exp_spec(dt*A);  w = (dt*x)*B;  h' = fma(a, h, w)      all binary32, in this order
- *   y  = sum_n C[n]*h'[n] + D*x                  (FP32 accumulation, tree order unspecified)
+ *   y  = (sum_n C[n]*h'[n] + D*x) [* z*sigmoid(z)]   (FP32 accumulation, tree order unspecified)
  *   E4M3 / INTb: s = max(amax_block(h') / top, FLT_MIN) with top = 448 / q_max, v = h' * (1/s);  otherwise v = h'
  *   state = encode(Q_u(v)) with u from `rule` at write index step_t (first write is step_t = 1)
  * exp_spec is the library's fixed binary32 exponential (clamp to [-87, 88], Cody-Waite reduction,
@@ -138,12 +145,13 @@ typedef struct {
     float* y;         uint64_t stride_y;    /* each [B, H, P]; written for every (t, l) slot of the ring */
     uint32_t ring;    /* number of distinct steps stored (>= 1; == n_steps when every step has its own inputs) */
     uint32_t reserved;
+    const float* z;   uint64_t stride_z;    /* each [B, H, P], or NULL: no gate */
 } ssdq_step_inputs;
 
 /* T-step decode driver (the open-loop replay of Appendix B run forward): for t = t_first ..
  * t_first + n_steps - 1 and l = 0 .. n_layers - 1, one ssd_state_update launch of layers[l] with
  * write index t and the inputs of slot (t, l), all on `stream`, no host synchronisation.  The
- * x / dt / Bm / Cm / y members of layers[l] are ignored (taken from `in`). */
+ * x / dt / Bm / Cm / y / z members of layers[l] are ignored (taken from `in`). */
 int ssd_decode_run(const ssdq_update_desc* layers, uint32_t n_layers, uint32_t t_first, uint32_t n_steps,
                    const ssdq_step_inputs* in, void* stream);
 

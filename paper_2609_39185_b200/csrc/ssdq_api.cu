@@ -68,6 +68,8 @@ int check_layer(const ssdq_update_desc* d) {
     if (!aligned16(d->state)) return fail(SSDQ_ERR_ALIGN, "state must be 16-byte aligned");
     if (d->a_per_state ? !aligned16(d->A) : !aligned4(d->A)) return fail(SSDQ_ERR_ALIGN, "A is misaligned");
     if (d->D && !aligned4(d->D)) return fail(SSDQ_ERR_ALIGN, "D is misaligned");
+    if (d->dt_bias && !aligned4(d->dt_bias)) return fail(SSDQ_ERR_ALIGN, "dt_bias is misaligned");
+    if (d->ngroups > 1 && d->nheads % d->ngroups != 0) return fail(SSDQ_ERR_SHAPE, "nheads must be a multiple of ngroups");
     if (format_scaled(d->format)) {
         if (!d->scales) return fail(SSDQ_ERR_NULL, "E4M3 and INTb stores need a scale array");
         if (!aligned4(d->scales)) return fail(SSDQ_ERR_ALIGN, "scales are misaligned");
@@ -82,9 +84,9 @@ int check_layer(const ssdq_update_desc* d) {
     return SSDQ_OK;
 }
 
-int check_step_ptrs(const float* x, const float* dt, const float* Bm, const float* Cm, const float* y) {
+int check_step_ptrs(const float* x, const float* dt, const float* Bm, const float* Cm, const float* y, const float* z = nullptr) {
     if (!x || !dt || !Bm || !Cm || !y) return fail(SSDQ_ERR_NULL, "x, dt, Bm, Cm and y are required");
-    if (!aligned4(x) || !aligned4(dt) || !aligned4(y)) return fail(SSDQ_ERR_ALIGN, "x, dt or y is misaligned");
+    if (!aligned4(x) || !aligned4(dt) || !aligned4(y) || !aligned4(z)) return fail(SSDQ_ERR_ALIGN, "x, dt, y or z is misaligned");
     if (!aligned16(Bm) || !aligned16(Cm)) return fail(SSDQ_ERR_ALIGN, "Bm and Cm must be 16-byte aligned");
     return SSDQ_OK;
 }
@@ -93,6 +95,9 @@ ssdq::UpdateParams make_params(const ssdq_update_desc* d, uint32_t step_t) {
     ssdq::UpdateParams p{};
     p.state = d->state; p.scales = d->scales;
     p.x = d->x; p.dt = d->dt; p.A = d->A; p.Bm = d->Bm; p.Cm = d->Cm; p.D = d->D; p.y = d->y;
+    p.dt_bias = d->dt_bias; p.z = d->z; p.dt_softplus = d->dt_softplus;
+    p.ngroups = d->ngroups > 1 ? d->ngroups : 1;
+    p.heads_per_group = d->nheads / p.ngroups;
     p.B = d->batch; p.H = d->nheads; p.P = d->headdim; p.N = d->dstate;
     p.n_items = d->batch * d->nheads;
     p.scale_block = d->scale_block;
@@ -198,7 +203,7 @@ int ssdq_thresholds_materialize(int rule, const ssdq_weyl* weyl, uint64_t sr_see
 int ssd_state_update(const ssdq_update_desc* d, uint32_t step_t, void* stream) {
     int rc = check_layer(d);
     if (rc != SSDQ_OK) return rc;
-    rc = check_step_ptrs(d->x, d->dt, d->Bm, d->Cm, d->y);
+    rc = check_step_ptrs(d->x, d->dt, d->Bm, d->Cm, d->y, d->z);
     if (rc != SSDQ_OK) return rc;
     const ssdq::UpdateParams p = make_params(d, step_t);
     return cuda_result(launch_update(p, d->format, d->rule, d->a_per_state != 0, static_cast<cudaStream_t>(stream)),
@@ -270,6 +275,7 @@ int ssd_decode_run(const ssdq_update_desc* layers, uint32_t n_layers, uint32_t t
             p.Bm = in->Bm + k * in->stride_B;
             p.Cm = in->Cm + k * in->stride_C;
             p.y = in->y + k * in->stride_y;
+            p.z = in->z ? in->z + k * in->stride_z : nullptr;
             const int rc = cuda_result(launch_update(p, layers[l].format, layers[l].rule, layers[l].a_per_state != 0, s),
                                        "state-update kernel");
             if (rc != SSDQ_OK) return rc;
@@ -312,7 +318,8 @@ int ssd_decode_run_host(const ssdq_update_desc* layers, uint32_t n_layers, uint3
     if (n_layers == 0 || host->ring == 0) return fail(SSDQ_ERR_SHAPE, "n_layers and host ring must be positive");
     if (staging->ring < 2 || staging->ring > kMaxStagingSlots) return fail(SSDQ_ERR_SHAPE, "staging ring must hold 2 to 8 slots");
     if (host->stride_x != staging->stride_x || host->stride_dt != staging->stride_dt || host->stride_B != staging->stride_B ||
-        host->stride_C != staging->stride_C || host->stride_y != staging->stride_y)
+        host->stride_C != staging->stride_C || host->stride_y != staging->stride_y || host->stride_z != staging->stride_z ||
+        (host->z == nullptr) != (staging->z == nullptr))
         return fail(SSDQ_ERR_SHAPE, "host and staging strides must be equal");
     if (!host->x || !host->dt || !host->Bm || !host->Cm || !host->y) return fail(SSDQ_ERR_NULL, "host x, dt, Bm, Cm and y are required");
     for (uint32_t l = 0; l < n_layers; ++l) {
@@ -352,6 +359,9 @@ int ssd_decode_run_host(const ssdq_update_desc* layers, uint32_t n_layers, uint3
                                  L * host->stride_B * sizeof(float), cudaMemcpyHostToDevice, hp->h2d));
         SSDQ_TRY(cudaMemcpyAsync(const_cast<float*>(staging->Cm) + dk * staging->stride_C, host->Cm + hk * host->stride_C,
                                  L * host->stride_C * sizeof(float), cudaMemcpyHostToDevice, hp->h2d));
+        if (host->z)
+            SSDQ_TRY(cudaMemcpyAsync(const_cast<float*>(staging->z) + dk * staging->stride_z, host->z + hk * host->stride_z,
+                                     L * host->stride_z * sizeof(float), cudaMemcpyHostToDevice, hp->h2d));
         SSDQ_TRY(cudaEventRecord(hp->loaded[sl], hp->h2d));
         // the fused updates of step i, once its inputs have landed and the slot's previous y has left
         SSDQ_TRY(cudaStreamWaitEvent(compute, hp->loaded[sl], 0));
@@ -364,6 +374,7 @@ int ssd_decode_run_host(const ssdq_update_desc* layers, uint32_t n_layers, uint3
             p.Bm = staging->Bm + k * staging->stride_B;
             p.Cm = staging->Cm + k * staging->stride_C;
             p.y = staging->y + k * staging->stride_y;
+            p.z = staging->z ? staging->z + k * staging->stride_z : nullptr;
             rc = cuda_result(launch_update(p, layers[l].format, layers[l].rule, layers[l].a_per_state != 0, compute),
                              "state-update kernel");
             if (rc != SSDQ_OK) return rc;

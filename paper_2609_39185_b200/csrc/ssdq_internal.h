@@ -16,8 +16,13 @@ struct UpdateParams {
     const float* Bm;
     const float* Cm;
     const float* D;
+    const float* dt_bias;    // [H] or null
+    const float* z;          // [B,H,P] or null: y <- y * silu(z)
     float* y;
     uint32_t B, H, P, N;
+    uint32_t dt_softplus;    // dt <- softplus_spec(dt + dt_bias)
+    uint32_t ngroups;        // B, C are [B, G, N]
+    uint32_t heads_per_group;
     uint32_t n_items;        // B * H
     uint32_t scale_block;    // scaled stores: 16 or N
     float scale_top;         // scaled stores: block scale = amax / scale_top (448 for E4M3, q_max for INTb)

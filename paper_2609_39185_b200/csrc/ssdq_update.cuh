@@ -193,8 +193,9 @@ __global__ void __launch_bounds__(kThreads) ssd_update_kernel(const UpdateParams
     // lane constants: B[n], C[n], decay(s), dt, D
     float Bv[EPL], Cv[EPL];
     {
-        const float4* Bp = reinterpret_cast<const float4*>(p.Bm + (size_t)b * N + n0);
-        const float4* Cp = reinterpret_cast<const float4*>(p.Cm + (size_t)b * N + n0);
+        const size_t grp = (size_t)b * p.ngroups + h / p.heads_per_group;
+        const float4* Bp = reinterpret_cast<const float4*>(p.Bm + grp * N + n0);
+        const float4* Cp = reinterpret_cast<const float4*>(p.Cm + grp * N + n0);
 #pragma unroll
         for (int i = 0; i < EPL / 4; ++i) {
             const float4 bb = __ldg(Bp + i), cc = __ldg(Cp + i);
@@ -202,7 +203,9 @@ __global__ void __launch_bounds__(kThreads) ssd_update_kernel(const UpdateParams
             Cv[4 * i] = cc.x; Cv[4 * i + 1] = cc.y; Cv[4 * i + 2] = cc.z; Cv[4 * i + 3] = cc.w;
         }
     }
-    const float dtv = __ldg(p.dt + item);
+    float dtv = __ldg(p.dt + item);
+    if (p.dt_bias) dtv = __fadd_rn(dtv, __ldg(p.dt_bias + h));
+    if (p.dt_softplus) dtv = softplus_spec(dtv);
     const float Dv = p.D ? __ldg(p.D + h) : 0.0f;
     float av[APS ? EPL : 1];
     if constexpr (APS) {
@@ -301,7 +304,8 @@ __global__ void __launch_bounds__(kThreads) ssd_update_kernel(const UpdateParams
             if (last_of_batch) {
                 const uint32_t kb = k - (k % LPR);                // first row of this batch of <= LPR rows
                 const uint32_t kk = kb + lis;
-                if (item_ok && kk <= k && kk < p.rps && (p_first + kk < p.P)) p.y[row_first + kk] = ykeep;
+                if (item_ok && kk <= k && kk < p.rps && (p_first + kk < p.P))
+                    p.y[row_first + kk] = p.z ? __fmul_rn(ykeep, silu(__ldg(p.z + row_first + kk))) : ykeep;
             }
         }
     }
@@ -367,8 +371,9 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
     }
     float Bv[EPL], Cv[EPL];
     {
-        const float4* Bp = reinterpret_cast<const float4*>(p.Bm + (size_t)b * N + n0);
-        const float4* Cp = reinterpret_cast<const float4*>(p.Cm + (size_t)b * N + n0);
+        const size_t grp = (size_t)b * p.ngroups + h / p.heads_per_group;
+        const float4* Bp = reinterpret_cast<const float4*>(p.Bm + grp * N + n0);
+        const float4* Cp = reinterpret_cast<const float4*>(p.Cm + grp * N + n0);
 #pragma unroll
         for (int i = 0; i < EPL / 4; ++i) {
             const float4 bb = __ldg(Bp + i), cc = __ldg(Cp + i);
@@ -376,7 +381,15 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
             Cv[4 * i] = cc.x; Cv[4 * i + 1] = cc.y; Cv[4 * i + 2] = cc.z; Cv[4 * i + 3] = cc.w;
         }
     }
-    const float dtv = __ldg(p.dt + item);
+    float dtv = __ldg(p.dt + item);
+    if (p.dt_bias) dtv = __fadd_rn(dtv, __ldg(p.dt_bias + h));
+    if (p.dt_softplus) dtv = softplus_spec(dtv);
+    // the lanes that will write y fetch their gate values now (row j = lane_in_slot / (LPR / 4) of each group of four)
+    const bool y_writer = (lis & (LPR / 4 - 1)) == 0;
+    float gate[RPS / 4];
+#pragma unroll
+    for (int g4 = 0; g4 < RPS / 4; ++g4)
+        gate[g4] = (p.z && y_writer) ? __ldg(p.z + row_first + g4 * 4 + lis / (LPR / 4)) : 0.0f;
     const float a = exp_spec(__fmul_rn(dtv, __ldg(p.A + h)));
     const float Dl = (p.D && lis == 0) ? __ldg(p.D + h) : 0.0f;     // the skip term enters the dot on one lane
 
@@ -431,7 +444,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
             if constexpr (RULE == RULE_SR) grp_row += N / 4;
         }
         const float tot = reduce4_over_slot<LPR>(dots[0], dots[1], dots[2], dots[3], lis);
-        if ((lis & (LPR / 4 - 1)) == 0) p.y[row_first + g4 * 4 + lis / (LPR / 4)] = tot;
+        if (y_writer) p.y[row_first + g4 * 4 + lis / (LPR / 4)] = p.z ? __fmul_rn(tot, silu(gate[g4])) : tot;
     }
 }
 

@@ -40,12 +40,14 @@ class UpdateDesc(ctypes.Structure):
                 ("state", _vp), ("scales", _vp), ("scale_block", _u32), ("format", _i32),
                 ("x", _vp), ("dt", _vp), ("A", _vp), ("Bm", _vp), ("Cm", _vp), ("D", _vp),
                 ("a_per_state", _u32), ("y", _vp), ("rule", _i32), ("weyl", Weyl), ("sr_seed", _u64),
-                ("layer", _u32), ("batch_index_base", _u32)]
+                ("layer", _u32), ("batch_index_base", _u32), ("dt_bias", _vp), ("z", _vp), ("dt_softplus", _u32),
+                ("ngroups", _u32)]
 
 
 class StepInputs(ctypes.Structure):
     _fields_ = [("x", _vp), ("stride_x", _u64), ("dt", _vp), ("stride_dt", _u64), ("Bm", _vp), ("stride_B", _u64),
-                ("Cm", _vp), ("stride_C", _u64), ("y", _vp), ("stride_y", _u64), ("ring", _u32), ("reserved", _u32)]
+                ("Cm", _vp), ("stride_C", _u64), ("y", _vp), ("stride_y", _u64), ("ring", _u32), ("reserved", _u32),
+                ("z", _vp), ("stride_z", _u64)]
 
 
 _lib = None
@@ -121,7 +123,7 @@ def thresholds_materialize(rule, n, step_t, *, weyl=None, sr_seed=0, layer=0, fi
 
 
 def make_desc(state, scales, fmt, *, A, D, rule, weyl=None, sr_seed=0, layer=0, scale_block=0, batch_index_base=0,
-              x=None, dt=None, Bm=None, Cm=None, y=None) -> UpdateDesc:
+              x=None, dt=None, Bm=None, Cm=None, y=None, dt_bias=None, dt_softplus=False, ngroups=1, z=None) -> UpdateDesc:
     """Describe one layer's problem.  `state` is a CUDA tensor of shape [B, H, P, N] holding the codes
     (uint8 for E4M3, int16/uint16/float16/bfloat16 for the 16-bit formats, float32 for the FP32 twin)."""
     B, H, P, N = state.shape
@@ -135,16 +137,18 @@ def make_desc(state, scales, fmt, *, A, D, rule, weyl=None, sr_seed=0, layer=0, 
     if weyl is not None:
         d.weyl = weyl
     d.sr_seed, d.layer, d.batch_index_base = sr_seed, layer, batch_index_base
+    d.dt_bias, d.z, d.dt_softplus, d.ngroups = _ptr(dt_bias), _ptr(z), int(bool(dt_softplus)), ngroups
     # keep the tensors alive as long as the descriptor
-    d._keep = (state, scales, A, D, x, dt, Bm, Cm, y)
+    d._keep = (state, scales, A, D, x, dt, Bm, Cm, y, dt_bias, z)
     return d
 
 
-def ssd_state_update(desc: UpdateDesc, step_t: int, *, x=None, dt=None, Bm=None, Cm=None, y=None):
+def ssd_state_update(desc: UpdateDesc, step_t: int, *, x=None, dt=None, Bm=None, Cm=None, y=None, z=None):
     """One fused decode step of one layer, in place on desc.state; y is written.  Per-step tensors may be
     given here (they overwrite the descriptor's pointers)."""
     if x is not None:
         desc.x, desc.dt, desc.Bm, desc.Cm, desc.y = _ptr(x), _ptr(dt), _ptr(Bm), _ptr(Cm), _ptr(y)
+        desc.z = _ptr(z)
     _check(lib().ssd_state_update(ctypes.byref(desc), step_t & 0xFFFFFFFF, _stream()))
 
 
@@ -161,8 +165,9 @@ def dequantize(codes, scales, fmt, out, scale_block=0):
     _check(lib().ssdq_dequantize(_ptr(codes), _ptr(scales), codes.numel(), fmt, scale_block, _ptr(out), _stream()))
 
 
-def make_step_inputs(x, dt, Bm, Cm, y) -> StepInputs:
-    """x [ring, L, B, H, P], dt [ring, L, B, H], Bm/Cm [ring, L, B, N], y [ring, L, B, H, P] CUDA float32."""
+def make_step_inputs(x, dt, Bm, Cm, y, z=None) -> StepInputs:
+    """x [ring, L, B, H, P], dt [ring, L, B, H], Bm/Cm [ring, L, B, (G,) N], y and optional gate z [ring, L, B, H, P];
+    float32, all on the device or (for ssd_decode_run_host's host side) all pinned host tensors."""
     s = StepInputs()
     s.ring = x.shape[0]
     s.x, s.stride_x = _ptr(x), x[0, 0].numel()
@@ -170,7 +175,9 @@ def make_step_inputs(x, dt, Bm, Cm, y) -> StepInputs:
     s.Bm, s.stride_B = _ptr(Bm), Bm[0, 0].numel()
     s.Cm, s.stride_C = _ptr(Cm), Cm[0, 0].numel()
     s.y, s.stride_y = _ptr(y), y[0, 0].numel()
-    s._keep = (x, dt, Bm, Cm, y)
+    if z is not None:
+        s.z, s.stride_z = _ptr(z), z[0, 0].numel()
+    s._keep = (x, dt, Bm, Cm, y, z)
     return s
 
 

@@ -40,11 +40,12 @@ class Pair:
     """One layer's state held twice: on the GPU (library) and on the host (oracle)."""
 
     def __init__(self, shape, fmt, rule, A, D, *, weyl_block=16, scale_block=0, layer=0, weyl_seed=0, sr_seed=0,
-                 batch_index_base=0, h0_codes=None, h0_scales=None):
+                 batch_index_base=0, h0_codes=None, h0_scales=None, dt_bias=None, dt_softplus=False, ngroups=1):
         self.shape, self.fmt, self.rule = shape, fmt, rule
         self.A, self.D = A, D
         self.kw = dict(layer=layer, weyl_seed=weyl_seed, weyl_block=weyl_block, sr_seed=sr_seed,
-                       batch_index_base=batch_index_base)
+                       batch_index_base=batch_index_base, dt_bias=dt_bias, dt_softplus=dt_softplus, ngroups=ngroups)
+        self.bias_d = to_dev(dt_bias)
         self.scale_block = scale_block
         if h0_codes is None:
             self.state_h, self.scales_h = oracle.new_state(shape, fmt, scale_block)
@@ -57,17 +58,19 @@ class Pair:
         weyl = ssdq.weyl_offsets_init(layer, weyl_seed, weyl_block)
         self.desc = ssdq.make_desc(self.state_d, self.scales_d, fmt, A=self.A_d, D=self.D_d, rule=rule, weyl=weyl,
                                    sr_seed=sr_seed, layer=layer, scale_block=scale_block,
-                                   batch_index_base=batch_index_base)
+                                   batch_index_base=batch_index_base, dt_bias=self.bias_d, dt_softplus=dt_softplus,
+                                   ngroups=ngroups)
         self.y_d = torch.empty(shape[:3], dtype=torch.float32, device="cuda")
 
-    def step_gpu(self, t, x, dt, Bm, Cm):
-        self._ins = [to_dev(v) for v in (x, dt, Bm, Cm)]
-        ssdq.ssd_state_update(self.desc, t, x=self._ins[0], dt=self._ins[1], Bm=self._ins[2], Cm=self._ins[3], y=self.y_d)
+    def step_gpu(self, t, x, dt, Bm, Cm, z=None):
+        self._ins = [to_dev(v) for v in (x, dt, Bm, Cm, z)]
+        ssdq.ssd_state_update(self.desc, t, x=self._ins[0], dt=self._ins[1], Bm=self._ins[2], Cm=self._ins[3], y=self.y_d,
+                              z=self._ins[4])
         return self.y_d
 
-    def step_oracle(self, t, x, dt, Bm, Cm):
+    def step_oracle(self, t, x, dt, Bm, Cm, z=None):
         return oracle.state_update(self.state_h, self.scales_h, self.fmt, self.scale_block, x, dt, self.A, Bm, Cm,
-                                   self.D, self.rule, t, **self.kw)
+                                   self.D, self.rule, t, z=z, **self.kw)
 
     def compare(self, t, x, dt, Bm, Cm, y_ref, y_absum=None):
         torch.cuda.synchronize()

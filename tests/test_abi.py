@@ -34,8 +34,8 @@ def test_every_declared_symbol_is_exported(lib):
 
 def test_struct_sizes_match_the_header():
     assert ctypes.sizeof(ssdq.Weyl) == 32
-    assert ctypes.sizeof(ssdq.UpdateDesc) == 160
-    assert ctypes.sizeof(ssdq.StepInputs) == 88
+    assert ctypes.sizeof(ssdq.UpdateDesc) == 184
+    assert ctypes.sizeof(ssdq.StepInputs) == 104
 
 
 def test_weyl_offsets_init_is_host_arithmetic(lib):

@@ -271,3 +271,38 @@ def test_host_buffer_driver_equals_device_driver(staging_slots, host_ring):
         for l in range(L):
             assert torch.equal(s1[l], s2[l])
         assert torch.equal(ys.cpu(), ys_h)
+
+
+@pytest.mark.parametrize("fmt", [ssdq.BF16, ssdq.FP16, ssdq.E4M3, ssdq.INT8])
+@pytest.mark.parametrize("rule", [ssdq.RTN, ssdq.WEYL])
+@pytest.mark.parametrize("shape,groups,aps", [((2, 8, 64, 128), 4, False), ((3, 6, 5, 64), 2, False), ((2, 12, 1, 16), 3, True)])
+def test_production_signature_options(fmt, rule, shape, groups, aps):
+    """dt_bias + in-kernel softplus, grouped B and C, z gate: state bit for bit, gated y to tolerance, on the tile
+    kernel's shape and on generic ones."""
+    B, H, P, N = shape
+    rng = np.random.default_rng(hash((fmt, rule) + shape) % 2**32)
+    f32 = np.float32
+    A = -np.exp(rng.uniform(-4, 1, (H, N) if aps else (H,))).astype(f32)
+    D = rng.normal(0, 0.1, H).astype(f32)
+    bias = rng.normal(-2, 1, H).astype(f32)
+    sb = N if oracle.has_block_scale(fmt) else 0
+    pair = Pair(shape, fmt, rule, A, D, weyl_block=16, scale_block=sb, dt_bias=bias, dt_softplus=True, ngroups=groups)
+    for t in range(1, 6):
+        x = rng.standard_normal((B, H, P)).astype(f32)
+        raw = rng.normal(-1, 2, (B, H)).astype(f32)
+        raw[0, 0] = 25.0                                            # beyond the softplus threshold
+        Bm = (rng.standard_normal((B, groups, N)) * 0.3).astype(f32)
+        Cm = rng.standard_normal((B, groups, N)).astype(f32)
+        z = rng.standard_normal((B, H, P)).astype(f32) * 2
+        y = pair.step_gpu(t, x, raw, Bm, Cm, z).cpu().numpy()
+        y_ref = pair.step_oracle(t, x, raw, Bm, Cm, z)
+        torch.cuda.synchronize()
+        assert np.array_equal(codes_to_host(pair.state_d, fmt), pair.state_h), t
+        if pair.scales_h is not None:
+            assert np.array_equal(pair.scales_d.cpu().numpy().view(np.uint32), pair.scales_h.view(np.uint32))
+        # tolerance: the ungated bound times |silu(z)|, plus the gate's own relative error
+        new_f32 = oracle.dequantize(pair.state_h, pair.scales_h, fmt, sb).reshape(shape).astype(np.float64)
+        Cexp = np.repeat(Cm, H // groups, axis=1).astype(np.float64)            # [B, H, N]
+        absum = np.einsum("bhpn,bhn->bhp", np.abs(new_f32), np.abs(Cexp)) + np.abs(D.astype(np.float64))[None, :, None] * np.abs(x)
+        gate = np.abs(z.astype(np.float64) / (1 + np.exp(-z.astype(np.float64))))
+        assert np.all(np.abs(y - y_ref) <= 1e-5 * absum * gate + 4e-6 * np.abs(y_ref) + 1e-30), t
