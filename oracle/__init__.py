@@ -75,6 +75,8 @@ def lib() -> ctypes.CDLL:
         L.oracle_softplus_spec.argtypes = [f32]
         L.oracle_quantize_store.restype = i32
         L.oracle_quantize_store.argtypes = [vp, vp, vp, u64, u32, i32, u32, i32, u32, u32, u32, u64, u64, u32]
+        L.oracle_replay_step.restype = i32
+        L.oracle_replay_step.argtypes = [vp, vp, u32, vp, vp, u64, u32, i32, u32, i32, u32, u32, u32, u64, u64, u32]
         L.oracle_dequantize.restype = None
         L.oracle_dequantize.argtypes = [vp, vp, u64, i32, u32, vp]
         L.oracle_num_threads.restype = i32
@@ -200,6 +202,19 @@ def quantize_store(src, fmt, rule, step_t, *, scale_block=0, layer=0, weyl_seed=
     if rc != 0:
         raise ValueError("oracle_quantize_store: undefined argument combination")
     return codes, scales
+
+
+def replay_step(w, a, rows_per_decay, codes, scales, fmt, rule, step_t, *, scale_block=0, layer=0, weyl_seed=0,
+                weyl_block=16, sr_seed=0, row_index_base=0):
+    """Open-loop replay h <- Q(a h + w), in place on codes [n_rows, row_len] (and scales); w float32 [n_rows, row_len],
+    a float32 [n_rows / rows_per_decay]."""
+    w, a = _f32(w), _f32(a)
+    n_rows, row_len = codes.shape
+    assert w.shape == codes.shape and a.size * rows_per_decay == n_rows and codes.flags.c_contiguous
+    rc = lib().oracle_replay_step(_ptr(w), _ptr(a), rows_per_decay, _ptr(codes), _ptr(scales), n_rows, row_len, fmt, scale_block,
+                                  rule, layer, weyl_seed, weyl_block, sr_seed, row_index_base, step_t)
+    if rc != 0:
+        raise ValueError("oracle_replay_step: undefined argument combination")
 
 
 def dequantize(codes, scales, fmt, scale_block=0):

@@ -458,6 +458,49 @@ int oracle_quantize_store(const float* src, void* dst_codes, float* dst_scales, 
     return 0;
 }
 
+// ---- open-loop replay of recorded traces (Appendix B "Open-loop replay"): h_t = Q(a_t h_{t-1} + w_t) ------
+// codes [n_rows, row_len] (and scales) are updated in place from w [n_rows, row_len] and one decay per
+// `rows_per_decay` consecutive rows (a [n_rows / rows_per_decay]; a head of P rows shares its decay).  FP32:
+// h' = fma(a, dequant(code), w); then block scale, threshold and Eq. 2 exactly as in the decode step.
+int oracle_replay_step(const float* w, const float* a, uint32_t rows_per_decay, void* codes, float* scales,
+                       uint64_t n_rows, uint32_t row_len, int fmt, uint32_t scale_block, int rule, uint32_t layer,
+                       uint32_t weyl_seed, uint32_t weyl_block, uint64_t sr_seed, uint64_t row_index_base, uint32_t step_t) {
+    if (has_block_scale(fmt) && (scale_block == 0 || row_len % scale_block != 0 || !scales)) return -1;
+    if (rule == RULE_WEYL && (weyl_block == 0 || row_len % weyl_block != 0)) return -1;
+    if (rows_per_decay == 0 || n_rows % rows_per_decay != 0) return -1;
+    const RuleParams rp{rule, layer, weyl_seed, weyl_block, sr_seed};
+    const uint32_t blk = has_block_scale(fmt) ? scale_block : row_len;
+#pragma omp parallel for schedule(static)
+    for (int64_t row = 0; row < (int64_t)n_rows; ++row) {
+        const float av = a[row / rows_per_decay];
+        std::vector<float> hp(row_len);
+        for (uint32_t i = 0; i < row_len; ++i) {
+            const uint64_t local = (uint64_t)row * row_len + i;
+            float hv = decode(load_code(codes, local, fmt), fmt);
+            if (has_block_scale(fmt)) hv = hv * scales[local / scale_block];
+            hp[i] = std::fmaf(av, hv, w[local]);
+        }
+        for (uint32_t s0 = 0; s0 < row_len; s0 += blk) {
+            float rinv = 1.0f;
+            if (has_block_scale(fmt)) {
+                float amax = 0.0f;
+                for (uint32_t i = s0; i < s0 + blk; ++i) amax = std::max(amax, std::fabs(hp[i]));
+                const float s = block_scale(amax, fmt);
+                rinv = 1.0f / s;
+                scales[((uint64_t)row * row_len + s0) / blk] = s;
+            }
+            for (uint32_t i = s0; i < s0 + blk; ++i) {
+                const uint64_t local = (uint64_t)row * row_len + i;
+                const uint64_t flat = row_index_base * row_len + local;
+                const float v = has_block_scale(fmt) ? hp[i] * rinv : hp[i];
+                const uint32_t U = threshold_u24(rp, flat, step_t);
+                store_code(codes, local, fmt, encode(round_on_grid(v, fmt, rule, U), fmt));
+            }
+        }
+    }
+    return 0;
+}
+
 // Dequantise a store back to FP32 (for error metrics and for reading results).
 void oracle_dequantize(const void* codes, const float* scales, uint64_t n, int fmt, uint32_t scale_block, float* out) {
     for (uint64_t i = 0; i < n; ++i) {

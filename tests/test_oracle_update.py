@@ -291,3 +291,30 @@ def test_full_signature_reduces_to_the_plain_step():
                     zz = z[:, h:h + 1].astype(np.float64)
                     want = yh.astype(np.float64) * zz / (1 + np.exp(-zz))
                     assert np.allclose(y[:, h:h + 1], want, rtol=2e-6, atol=1e-7)
+
+
+# ---- open-loop replay and checkpointed rounding --------------------------------------------------
+@pytest.mark.parametrize("fmt", [FP16, BF16, E4M3, oracle.INT8])
+@pytest.mark.parametrize("rule", [RTN, SR, WEYL, SR_HASH])
+def test_replay_of_the_decomposed_step_reproduces_the_decode_step(fmt, rule):
+    """Appendix B "Open-loop replay": w_t = dt_t x_t (outer) B_t is rank one per head and a_t comes from the step
+    size.  Feeding exactly those a and w to the replay gives the state of the decode step, bit for bit."""
+    rng = np.random.default_rng(40 + fmt)
+    Bsz, H, P, N = 2, 3, 4, 32
+    f32 = np.float32
+    sb = 16 if oracle.has_block_scale(fmt) else 0
+    A = -np.exp(rng.uniform(-3, 1, H)).astype(f32)
+    st1, sc1 = oracle.new_state((Bsz, H, P, N), fmt, sb)
+    st2, sc2 = st1.reshape(-1, N).copy(), None if sc1 is None else sc1.copy()
+    for t in range(1, 7):
+        x = rng.standard_normal((Bsz, H, P)).astype(f32)
+        dt = np.log1p(np.exp(rng.normal(-2, 0.5, (Bsz, H)))).astype(f32)
+        Bm = rng.standard_normal((Bsz, N)).astype(f32)
+        Cm = rng.standard_normal((Bsz, N)).astype(f32)
+        oracle.state_update(st1, sc1, fmt, sb, x, dt, A, Bm, Cm, None, rule, t, layer=1, weyl_block=16, sr_seed=3)
+        a = oracle.exp_spec((dt * A[None, :]).astype(f32).ravel())
+        w = ((dt[:, :, None] * x).astype(f32)[..., None] * Bm[:, None, None, :]).astype(f32)
+        oracle.replay_step(w.reshape(-1, N), a, P, st2, sc2, fmt, rule, t, scale_block=sb, layer=1, weyl_block=16, sr_seed=3)
+        assert np.array_equal(st1.reshape(-1, N), st2)
+        if sc1 is not None:
+            assert np.array_equal(sc1, sc2)
