@@ -131,6 +131,16 @@ int quantize_store(const float* src, void* dst_codes, float* dst_scales, uint64_
                    uint32_t scale_block, int format, int rule, const ssdq_weyl* weyl, uint64_t sr_seed,
                    uint32_t layer, uint64_t row_index_base, uint32_t step_t, void* stream);
 
+/* Open-loop replay of recorded traces (Appendix B "Open-loop replay"): h_t = Q(a_t h_{t-1} + w_t), in place on a
+ * store.  w [n_rows, row_len] DEVICE floats (16-byte aligned) are the recorded writes, decay [n_rows / rows_per_decay]
+ * the recorded decays (rows_per_decay consecutive rows -- a head of P rows -- share one); codes / scales, the rule,
+ * its indices and step_t are those of quantize_store.  h' = fma(a, dequant(code), w) in binary32, then block scale,
+ * threshold and Eq. 2 exactly as in ssd_state_update (whose state it reproduces bit for bit when fed a = exp_spec(dt*A)
+ * and w = (dt*x)*B). */
+int ssd_replay_step(const float* w, const float* decay, uint32_t rows_per_decay, void* codes, float* scales, uint64_t n_rows,
+                    uint32_t row_len, uint32_t scale_block, int format, int rule, const ssdq_weyl* weyl, uint64_t sr_seed,
+                    uint32_t layer, uint64_t row_index_base, uint32_t step_t, void* stream);
+
 /* Inverse view of a store: out[i] = decode(code[i]) (* scale[i / scale_block] for E4M3), DEVICE. */
 int ssdq_dequantize(const void* codes, const float* scales, uint64_t n, int format, uint32_t scale_block,
                     float* out, void* stream);
@@ -154,6 +164,15 @@ typedef struct {
  * x / dt / Bm / Cm / y / z members of layers[l] are ignored (taken from `in`). */
 int ssd_decode_run(const ssdq_update_desc* layers, uint32_t n_layers, uint32_t t_first, uint32_t n_steps,
                    const ssdq_step_inputs* in, void* stream);
+
+/* Periodic checkpointing (Section 6.5 "Periodic checkpointing"; Appendix B "Decode regime", CC = 8): the state lives in
+ * full precision between checkpoints and only every `every`-th write, counted from t_first, is rounded into the store.
+ * work_fp32[l] is a caller-owned DEVICE buffer [B, H, P, N] of floats holding layer l's working state (on entry: the
+ * dequantised store, or zeros for h_0 = 0).  Per step and layer: one FP32 update launch; on checkpoint steps also
+ * quantize_store (work -> layers[l].state under the layer's rule at write index t) and ssdq_dequantize (store -> work).
+ * With every == 1 the stores and y equal those of ssd_decode_run.  dstate <= 128. */
+int ssd_decode_run_checkpointed(const ssdq_update_desc* layers, float* const* work_fp32, uint32_t n_layers, uint32_t every,
+                                uint32_t t_first, uint32_t n_steps, const ssdq_step_inputs* in, void* stream);
 
 /* The same driver for callers whose per-step inputs and outputs live in HOST memory (the usual case when the
  * rest of the model runs elsewhere): `host` describes HOST arrays (page-locked memory for full speed) laid out like

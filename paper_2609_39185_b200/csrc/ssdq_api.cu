@@ -234,6 +234,82 @@ int quantize_store(const float* src, void* dst_codes, float* dst_scales, uint64_
     return cuda_result(ssdq::launch_quantize(p, kernel_format(format), rule, static_cast<cudaStream_t>(stream)), "quantize kernel");
 }
 
+int ssd_replay_step(const float* w, const float* decay, uint32_t rows_per_decay, void* codes, float* scales, uint64_t n_rows,
+                    uint32_t row_len, uint32_t scale_block, int format, int rule, const ssdq_weyl* weyl, uint64_t sr_seed,
+                    uint32_t layer, uint64_t row_index_base, uint32_t step_t, void* stream) {
+    if (!format_known(format)) return fail(SSDQ_ERR_UNSUPPORTED, "unknown format %d", format);
+    if (rule < SSDQ_RTN || rule > SSDQ_SR_HASH) return fail(SSDQ_ERR_UNSUPPORTED, "unknown rule %d", rule);
+    if (!dstate_supported(format, row_len)) return fail(SSDQ_ERR_UNSUPPORTED, "row_len %u is not supported for format %d", row_len, format);
+    if (rows_per_decay == 0 || n_rows % rows_per_decay != 0) return fail(SSDQ_ERR_SHAPE, "n_rows must be a multiple of rows_per_decay");
+    if (n_rows == 0) return SSDQ_OK;
+    if (!w || !decay || !codes) return fail(SSDQ_ERR_NULL, "w, decay and codes are required");
+    if (!aligned16(w) || !aligned16(codes) || !aligned4(decay)) return fail(SSDQ_ERR_ALIGN, "w and codes must be 16-byte aligned");
+    ssdq::QuantParams p{};
+    if (format_scaled(format)) {
+        if (!scales) return fail(SSDQ_ERR_NULL, "E4M3 and INTb stores need a scale array");
+        if (!(scale_block == 16 || scale_block == row_len)) return fail(SSDQ_ERR_SHAPE, "scale_block must be 16 or row_len");
+    }
+    if (rule == SSDQ_WEYL && format != SSDQ_FP32) {
+        if (!weyl) return fail(SSDQ_ERR_NULL, "weyl descriptor is NULL");
+        if (!(weyl->block == 16 || weyl->block == row_len)) return fail(SSDQ_ERR_SHAPE, "weyl.block must be 16 or row_len");
+        p.weyl = weyl_const(*weyl);
+    }
+    p.src = w; p.decay = decay; p.rows_per_decay = rows_per_decay; p.codes = codes; p.scales = scales; p.n_rows = n_rows;
+    p.row_len = row_len; p.scale_block = scale_block; p.scale_top = scale_top(format); p.step_t = step_t; p.layer = layer;
+    p.row_base = row_index_base; p.sr_seed = sr_seed;
+    return cuda_result(ssdq::launch_quantize(p, kernel_format(format), format == SSDQ_FP32 ? (int)SSDQ_RTN : rule,
+                                             static_cast<cudaStream_t>(stream)), "replay kernel");
+}
+
+int ssd_decode_run_checkpointed(const ssdq_update_desc* layers, float* const* work_fp32, uint32_t n_layers, uint32_t every,
+                                uint32_t t_first, uint32_t n_steps, const ssdq_step_inputs* in, void* stream) {
+    if (!layers || !in || !work_fp32) return fail(SSDQ_ERR_NULL, "layers, work_fp32 and in are required");
+    if (n_layers == 0 || in->ring == 0 || every == 0) return fail(SSDQ_ERR_SHAPE, "n_layers, ring and every must be positive");
+    for (uint32_t l = 0; l < n_layers; ++l) {
+        const int rc = check_layer(&layers[l]);
+        if (rc != SSDQ_OK) return rc;
+        if (layers[l].format == SSDQ_FP32) return fail(SSDQ_ERR_UNSUPPORTED, "the store of a checkpointed run must be a quantised format");
+        if (!work_fp32[l] || !aligned16(work_fp32[l])) return fail(SSDQ_ERR_ALIGN, "work_fp32[l] must be a 16-byte aligned device buffer");
+        if (layers[l].dstate > 128) return fail(SSDQ_ERR_UNSUPPORTED, "checkpointed runs need dstate <= 128 (FP32 working state)");
+    }
+    const uint32_t slots = n_steps < in->ring ? n_steps : in->ring;
+    for (uint32_t sl = 0; sl < slots; ++sl)
+        for (uint32_t l = 0; l < n_layers; ++l) {
+            const uint64_t k = (uint64_t)sl * n_layers + l;
+            const int rc = check_step_ptrs(in->x + k * in->stride_x, in->dt + k * in->stride_dt, in->Bm + k * in->stride_B,
+                                           in->Cm + k * in->stride_C, in->y + k * in->stride_y, in->z ? in->z + k * in->stride_z : nullptr);
+            if (rc != SSDQ_OK) return rc;
+        }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    for (uint32_t i = 0; i < n_steps; ++i) {
+        const uint32_t t = t_first + i;
+        for (uint32_t l = 0; l < n_layers; ++l) {
+            const ssdq_update_desc& d = layers[l];
+            const uint64_t k = (uint64_t)(i % in->ring) * n_layers + l;
+            // the update itself runs on the FP32 working state, unrounded
+            ssdq::UpdateParams p = make_params(&d, t);
+            p.state = work_fp32[l]; p.scales = nullptr; p.scale_block = 0;
+            p.x = in->x + k * in->stride_x;
+            p.dt = in->dt + k * in->stride_dt;
+            p.Bm = in->Bm + k * in->stride_B;
+            p.Cm = in->Cm + k * in->stride_C;
+            p.y = in->y + k * in->stride_y;
+            p.z = in->z ? in->z + k * in->stride_z : nullptr;
+            int rc = cuda_result(launch_update(p, SSDQ_FP32, SSDQ_RTN, d.a_per_state != 0, s), "state-update kernel");
+            if (rc != SSDQ_OK) return rc;
+            if ((i + 1) % every != 0) continue;
+            // every `every`-th write is rounded into the store (Eq. 2 under the layer's rule) and read back
+            const uint64_t n_rows = (uint64_t)d.batch * d.nheads * d.headdim;
+            rc = quantize_store(work_fp32[l], d.state, d.scales, n_rows, d.dstate, d.scale_block, d.format, d.rule, &d.weyl,
+                                d.sr_seed, d.layer, (uint64_t)d.batch_index_base * d.nheads * d.headdim, t, stream);
+            if (rc != SSDQ_OK) return rc;
+            rc = ssdq_dequantize(d.state, d.scales, n_rows * d.dstate, d.format, d.scale_block, work_fp32[l], stream);
+            if (rc != SSDQ_OK) return rc;
+        }
+    }
+    return SSDQ_OK;
+}
+
 int ssdq_dequantize(const void* codes, const float* scales, uint64_t n, int format, uint32_t scale_block, float* out,
                     void* stream) {
     if (!format_known(format)) return fail(SSDQ_ERR_UNSUPPORTED, "unknown format %d", format);

@@ -36,9 +36,11 @@ struct UpdateParams {
     uint64_t sr_seed;
 };
 
-// Parameters of quantize_store / dequantize / thresholds.
+// Parameters of quantize_store / replay / dequantize / thresholds.
 struct QuantParams {
     const float* src;
+    const float* decay;       // replay only: one decay per rows_per_decay consecutive rows
+    uint32_t rows_per_decay;
     void* codes;
     float* scales;
     uint64_t n_rows;
@@ -59,7 +61,7 @@ cudaError_t launch_update_e4m3(const UpdateParams& p, int rule, bool a_per_state
 cudaError_t launch_update_fp32(const UpdateParams& p, int rule, bool a_per_state, cudaStream_t s);
 cudaError_t launch_update_int8(const UpdateParams& p, int rule, bool a_per_state, cudaStream_t s);
 
-cudaError_t launch_quantize(const QuantParams& p, int fmt, int rule, cudaStream_t s);
+cudaError_t launch_quantize(const QuantParams& p, int fmt, int rule, cudaStream_t s);   // p.decay != null: replay step
 cudaError_t launch_dequantize(const void* codes, const float* scales, uint64_t n, int fmt, uint32_t scale_block,
                               float* out, cudaStream_t s);
 cudaError_t launch_thresholds(int rule, const WeylConst& w, uint64_t sr_seed, uint32_t layer, uint64_t first_flat,

@@ -5,7 +5,9 @@
 namespace ssdq {
 
 // One slot (LPR lanes) per row, grid-stride over rows; same lane-to-entry mapping as the fused kernel.
-template <int FMT, int RULE, int LPR>
+// REPLAY: the open-loop replay step h <- Q(a h + src) (Appendix B "Open-loop replay"): the old codes are
+// dequantised, multiplied by the row's recorded decay and the recorded write is added with one fused multiply-add.
+template <int FMT, int RULE, int LPR, bool REPLAY>
 __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantParams p) {
     constexpr int EPL = Fmt<FMT>::kEpl;
     constexpr int N = LPR * EPL;
@@ -28,6 +30,23 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantParams p)
             float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
             if (ok) f = reinterpret_cast<const float4*>(p.src + row * N + lis * EPL)[i];
             v[4 * i] = f.x; v[4 * i + 1] = f.y; v[4 * i + 2] = f.z; v[4 * i + 3] = f.w;
+        }
+        if constexpr (REPLAY) {
+            float h[EPL];
+            uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+            float a = 0.0f, s_old = 0.0f;
+            if (ok) {
+                raw = reinterpret_cast<const uint4*>(p.codes)[row * LPR + lis];
+                a = __ldg(p.decay + row / p.rows_per_decay);
+                if constexpr (Fmt<FMT>::kScaled) s_old = row_scale ? p.scales[row] : p.scales[row * (N / 16) + lis];
+            }
+            unpack_lane<FMT>(raw, h);
+#pragma unroll
+            for (int j = 0; j < EPL; ++j) {
+                float hin = h[j];
+                if constexpr (Fmt<FMT>::kScaled) hin = __fmul_rn(hin, s_old);
+                v[j] = __fmaf_rn(a, hin, v[j]);
+            }
         }
         if constexpr (Fmt<FMT>::kScaled) {
             float amax = 0.0f;
@@ -62,7 +81,8 @@ static cudaError_t launch_quantize_one(const QuantParams& p, cudaStream_t s) {
     uint64_t grid = (p.n_rows + NSLOT - 1) / NSLOT;
     if (grid > 148u * 64u) grid = 148u * 64u;
     if (grid == 0) return cudaSuccess;
-    quantize_kernel<FMT, RULE, LPR><<<(unsigned)grid, kThreads, 0, s>>>(p);
+    if (p.decay) quantize_kernel<FMT, RULE, LPR, true><<<(unsigned)grid, kThreads, 0, s>>>(p);
+    else quantize_kernel<FMT, RULE, LPR, false><<<(unsigned)grid, kThreads, 0, s>>>(p);
     return cudaGetLastError();
 }
 

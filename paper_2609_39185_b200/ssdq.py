@@ -18,7 +18,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libssdq.so")
 
 EXPORTS = ("weyl_offsets_init", "ssdq_thresholds_materialize", "ssd_state_update", "quantize_store",
-           "ssdq_dequantize", "ssd_decode_run", "ssd_decode_run_host", "ssdq_state_error_workspace_bytes", "ssdq_state_error",
+           "ssdq_dequantize", "ssd_decode_run", "ssd_decode_run_host", "ssd_replay_step", "ssd_decode_run_checkpointed", "ssdq_state_error_workspace_bytes", "ssdq_state_error",
            "ssdq_state_error_static", "ssdq_readout_kl", "ssdq_last_error", "ssdq_launch_count")
 
 _u32, _u64, _i32, _vp = ctypes.c_uint32, ctypes.c_uint64, ctypes.c_int32, ctypes.c_void_p
@@ -74,6 +74,12 @@ def lib() -> ctypes.CDLL:
         L.ssdq_dequantize.argtypes = [_vp, _vp, _u64, ctypes.c_int, _u32, _vp, _vp]
         L.ssd_decode_run.restype = ctypes.c_int
         L.ssd_decode_run.argtypes = [ctypes.POINTER(UpdateDesc), _u32, _u32, _u32, ctypes.POINTER(StepInputs), _vp]
+        L.ssd_replay_step.restype = ctypes.c_int
+        L.ssd_replay_step.argtypes = [_vp, _vp, _u32, _vp, _vp, _u64, _u32, _u32, ctypes.c_int, ctypes.c_int, ctypes.POINTER(Weyl),
+                                      _u64, _u32, _u64, _u32, _vp]
+        L.ssd_decode_run_checkpointed.restype = ctypes.c_int
+        L.ssd_decode_run_checkpointed.argtypes = [ctypes.POINTER(UpdateDesc), ctypes.POINTER(_vp), _u32, _u32, _u32, _u32,
+                                                  ctypes.POINTER(StepInputs), _vp]
         L.ssd_decode_run_host.restype = ctypes.c_int
         L.ssd_decode_run_host.argtypes = [ctypes.POINTER(UpdateDesc), _u32, _u32, _u32, ctypes.POINTER(StepInputs),
                                           ctypes.POINTER(StepInputs), _vp]
@@ -232,6 +238,24 @@ def ssd_decode_run_host(layer_descs, t_first: int, n_steps: int, host_io: StepIn
     arr = (UpdateDesc * len(layer_descs))(*layer_descs)
     _check(lib().ssd_decode_run_host(arr, len(layer_descs), t_first & 0xFFFFFFFF, n_steps, ctypes.byref(host_io),
                                      ctypes.byref(staging), _stream()))
+
+
+def replay_step(w, decay, rows_per_decay, codes, scales, fmt, rule, step_t, *, weyl=None, sr_seed=0, layer=0, scale_block=0,
+                row_index_base=0):
+    """Open-loop replay h <- Q(decay * h + w) in place on `codes` [n_rows, row_len] (and `scales`)."""
+    n_rows, row_len = codes.shape
+    wp = ctypes.byref(weyl) if weyl is not None else None
+    _check(lib().ssd_replay_step(_ptr(w), _ptr(decay), rows_per_decay, _ptr(codes), _ptr(scales), n_rows, row_len, scale_block,
+                                 fmt, rule, wp, sr_seed, layer, row_index_base, step_t & 0xFFFFFFFF, _stream()))
+
+
+def ssd_decode_run_checkpointed(layer_descs, work_states, every: int, t_first: int, n_steps: int, step_inputs: StepInputs):
+    """Decode with the state in FP32 between checkpoints; every `every`-th write is rounded into each layer's store.
+    work_states: one float32 CUDA tensor [B, H, P, N] per layer."""
+    arr = (UpdateDesc * len(layer_descs))(*layer_descs)
+    ptrs = (_vp * len(work_states))(*[w.data_ptr() for w in work_states])
+    _check(lib().ssd_decode_run_checkpointed(arr, ptrs, len(layer_descs), every, t_first & 0xFFFFFFFF, n_steps,
+                                             ctypes.byref(step_inputs), _stream()))
 
 
 def launch_count() -> int:

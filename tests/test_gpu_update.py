@@ -306,3 +306,86 @@ def test_production_signature_options(fmt, rule, shape, groups, aps):
         absum = np.einsum("bhpn,bhn->bhp", np.abs(new_f32), np.abs(Cexp)) + np.abs(D.astype(np.float64))[None, :, None] * np.abs(x)
         gate = np.abs(z.astype(np.float64) / (1 + np.exp(-z.astype(np.float64))))
         assert np.all(np.abs(y - y_ref) <= 1e-5 * absum * gate + 4e-6 * np.abs(y_ref) + 1e-30), t
+
+
+@pytest.mark.parametrize("fmt", [ssdq.FP16, ssdq.BF16, ssdq.E4M3, ssdq.INT8])
+@pytest.mark.parametrize("rule", RULES)
+def test_replay_step_matches_oracle_and_the_decode_step(fmt, rule):
+    """ssd_replay_step on recorded (a, w) traces: equal to the oracle's replay, and -- fed a = exp_spec(dt A) and
+    w = (dt x) B from the host -- equal to the fused decode step's state."""
+    rng = np.random.default_rng(70 + fmt)
+    B, H, P, N = 3, 5, 8, 128
+    f32 = np.float32
+    sb = N if oracle.has_block_scale(fmt) else 0
+    A = -np.exp(rng.uniform(-3, 1, H)).astype(f32)
+    pair = Pair((B, H, P, N), fmt, rule, A, None, weyl_block=16, scale_block=sb, layer=2, sr_seed=5, batch_index_base=4)
+    codes_h, scales_h = pair.state_h.reshape(-1, N).copy(), None if pair.scales_h is None else pair.scales_h.copy()
+    codes_d, scales_d = codes_to_dev(codes_h, fmt), to_dev(scales_h)
+    weyl = ssdq.weyl_offsets_init(2, 0, 16)
+    base = 4 * H * P
+    for t in range(1, 6):
+        x = rng.standard_normal((B, H, P)).astype(f32)
+        dt = np.log1p(np.exp(rng.normal(-2, 0.5, (B, H)))).astype(f32)
+        Bm = rng.standard_normal((B, N)).astype(f32)
+        Cm = rng.standard_normal((B, N)).astype(f32)
+        pair.step_gpu(t, x, dt, Bm, Cm)
+        a = oracle.exp_spec((dt * A[None, :]).astype(f32).ravel())
+        w = ((dt[:, :, None] * x).astype(f32)[..., None] * Bm[:, None, None, :]).astype(f32).reshape(-1, N)
+        ssdq.replay_step(to_dev(w), to_dev(a), P, codes_d, scales_d, fmt, rule, t, weyl=weyl, sr_seed=5, layer=2,
+                         scale_block=sb, row_index_base=base)
+        oracle.replay_step(w, a, P, codes_h, scales_h, fmt, rule, t, scale_block=sb, layer=2, weyl_block=16, sr_seed=5,
+                           row_index_base=base)
+        torch.cuda.synchronize()
+        assert np.array_equal(codes_to_host(codes_d, fmt), codes_h), t
+        assert np.array_equal(codes_to_host(pair.state_d, fmt).reshape(-1, N), codes_h), t
+        if scales_h is not None:
+            assert np.array_equal(scales_d.cpu().numpy().view(np.uint32), scales_h.view(np.uint32))
+
+
+@pytest.mark.parametrize("fmt", [ssdq.BF16, ssdq.E4M3, ssdq.INT8])
+@pytest.mark.parametrize("rule", [ssdq.RTN, ssdq.WEYL, ssdq.SR])
+def test_checkpointed_rounding(fmt, rule):
+    """Only every k-th write is rounded (CC = k).  k = 1 reproduces the plain driver; k = 4 equals the oracle's FP32
+    update with a quantise / dequantise round trip at every fourth write."""
+    from dataclasses import replace
+    cfg = replace(workloads.CONFIGS[4], batch=2, nheads=4, fmt=fmt)
+    sb, wb = cfg.scale_block if oracle.has_block_scale(fmt) else 0, cfg.weyl_block
+    T = 12
+    A, D = workloads.layer_params(cfg)
+    ins = [workloads.step_inputs(cfg, t) for t in range(1, T + 1)]
+    stack = lambda i: to_dev(np.stack([ins[t][i][None] for t in range(T)]))
+    xs, dts, Bs, Cs = (stack(i) for i in range(4))
+
+    def fresh():
+        st_h, sc_h = oracle.new_state(cfg.state_shape, fmt, sb)
+        st, sc = codes_to_dev(st_h, fmt), to_dev(sc_h)
+        desc = ssdq.make_desc(st, sc, fmt, A=to_dev(A), D=to_dev(D), rule=rule, weyl=ssdq.weyl_offsets_init(0, 0, wb), sr_seed=1,
+                              scale_block=sb)
+        return st, sc, desc
+
+    s1, c1, d1 = fresh()
+    y1 = torch.zeros_like(xs)
+    ssdq.ssd_decode_run([d1], 1, T, ssdq.make_step_inputs(xs, dts, Bs, Cs, y1))
+    s2, c2, d2 = fresh()
+    y2 = torch.zeros_like(xs)
+    work = torch.zeros(cfg.state_shape, dtype=torch.float32, device="cuda")
+    ssdq.ssd_decode_run_checkpointed([d2], [work], 1, 1, T, ssdq.make_step_inputs(xs, dts, Bs, Cs, y2))
+    torch.cuda.synchronize()
+    assert torch.equal(s1, s2) and (c1 is None or torch.equal(c1, c2))
+    assert torch.allclose(y1, y2, rtol=0, atol=1e-5 * float(y1.abs().max()))
+    # k = 4 against the oracle
+    s3, c3, d3 = fresh()
+    y3 = torch.zeros_like(xs)
+    work.zero_()
+    ssdq.ssd_decode_run_checkpointed([d3], [work], 4, 1, T, ssdq.make_step_inputs(xs, dts, Bs, Cs, y3))
+    w_h = np.zeros(cfg.state_shape, np.uint32)
+    N = cfg.dstate
+    for t in range(1, T + 1):
+        x, dt, Bm, Cm = ins[t - 1]
+        oracle.state_update(w_h, None, oracle.FP32, 0, x, dt, A, Bm, Cm, D, oracle.RTN, t)
+        if t % 4 == 0:
+            codes, scales = oracle.quantize_store(w_h.view(np.float32).reshape(-1, N), fmt, rule, t, scale_block=sb, weyl_block=wb, sr_seed=1)
+            w_h = oracle.dequantize(codes, scales, fmt, sb).reshape(cfg.state_shape).view(np.uint32).copy()
+    torch.cuda.synchronize()
+    assert np.array_equal(codes_to_host(s3, fmt).reshape(-1, N), codes)
+    assert np.array_equal(work.cpu().numpy().view(np.uint32), w_h)
