@@ -332,11 +332,27 @@ __device__ __forceinline__ float reduce4_over_slot(float d0, float d1, float d2,
     return k;
 }
 
+// cp.async.wait_group needs an immediate: allow at most RPS - 1 - k groups (the rows after k) to be pending.
+template <int RPS>
+__device__ __forceinline__ void cp_async_wait_rows(int k) {
+    switch (RPS - 1 - k) {
+        case 0: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;
+        case 1: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
+        case 2: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
+        case 3: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
+        case 4: asm volatile("cp.async.wait_group 4;" ::: "memory"); break;
+        case 5: asm volatile("cp.async.wait_group 5;" ::: "memory"); break;
+        case 6: asm volatile("cp.async.wait_group 6;" ::: "memory"); break;
+        default: asm volatile("cp.async.wait_group 7;" ::: "memory"); break;
+    }
+}
+
 // The tile kernel: the same computation for the shapes that dominate (one decay per head, a head of
 // P = (kThreads / LPR) * RPS rows), one CTA per (b, h).  A head's state is one contiguous tile (16 KB for
 // 64 x 128 two-byte codes); every lane issues all RPS of its 128-bit state loads, the x row and its
 // constants before touching any of them, then walks its rows four at a time.  No guards, no idle lanes.
-template <int FMT, int RULE, int LPR, int RPS>
+// EXTRAS: any of dt_bias, in-kernel softplus, B/C groups or the z gate is in use (the plain step pays nothing for them).
+template <int FMT, int RULE, int LPR, int RPS, bool EXTRAS>
 __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateParams p) {
     constexpr int EPL = Fmt<FMT>::kEpl;
     constexpr int N = LPR * EPL;
@@ -346,18 +362,25 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
 
     const uint32_t lis = threadIdx.x % LPR;
     const uint32_t slot = threadIdx.x / LPR;
-    const uint32_t item = blockIdx.x;
-    const uint32_t b = item / p.H;
-    const uint32_t h = item - b * p.H;
+    const uint32_t h = blockIdx.x;                  // grid = (H, B): no index division
+    const uint32_t b = blockIdx.y;
+    const uint32_t item = b * p.H + h;
     const uint32_t n0 = lis * EPL;
     const uint64_t row_first = (uint64_t)item * (NSLOT * RPS) + slot * RPS;
     const bool row_scale = Fmt<FMT>::kScaled && (p.scale_block == (uint32_t)N);
 
     // every load of the CTA is issued here
+    // The state tile goes global -> shared with asynchronous 16-byte copies, one commit group per row: the bytes in
+    // flight cost no registers (more CTAs per SM, hence more of them), and row k can be consumed as soon as it has
+    // landed while the later rows are still on their way.  Each lane reads back only what it copied itself, so
+    // cp.async.wait_group is all the synchronisation needed.
+    __shared__ uint4 tile[RPS][kThreads];
     uint4* sp = reinterpret_cast<uint4*>(p.state) + row_first * LPR + lis;
-    uint4 raw[RPS];
 #pragma unroll
-    for (int k = 0; k < RPS; ++k) raw[k] = sp[k * LPR];
+    for (int k = 0; k < RPS; ++k) {
+        const uint32_t dst = (uint32_t)__cvta_generic_to_shared(&tile[k][threadIdx.x]);
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n cp.async.commit_group;" ::"r"(dst), "l"(sp + k * LPR) : "memory");
+    }
     float xv[RPS];
     float sc[Fmt<FMT>::kScaled ? RPS : 1];
 #pragma unroll
@@ -371,7 +394,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
     }
     float Bv[EPL], Cv[EPL];
     {
-        const size_t grp = (size_t)b * p.ngroups + h / p.heads_per_group;
+        const size_t grp = (!EXTRAS || p.ngroups == 1) ? (size_t)b : (size_t)b * p.ngroups + h / p.heads_per_group;
         const float4* Bp = reinterpret_cast<const float4*>(p.Bm + grp * N + n0);
         const float4* Cp = reinterpret_cast<const float4*>(p.Cm + grp * N + n0);
 #pragma unroll
@@ -382,14 +405,16 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
         }
     }
     float dtv = __ldg(p.dt + item);
-    if (p.dt_bias) dtv = __fadd_rn(dtv, __ldg(p.dt_bias + h));
-    if (p.dt_softplus) dtv = softplus_spec(dtv);
+    if constexpr (EXTRAS) {
+        if (p.dt_bias) dtv = __fadd_rn(dtv, __ldg(p.dt_bias + h));
+        if (p.dt_softplus) dtv = softplus_spec(dtv);
+    }
     // the lanes that will write y fetch their gate values now (row j = lane_in_slot / (LPR / 4) of each group of four)
     const bool y_writer = (lis & (LPR / 4 - 1)) == 0;
     float gate[RPS / 4];
 #pragma unroll
     for (int g4 = 0; g4 < RPS / 4; ++g4)
-        gate[g4] = (p.z && y_writer) ? __ldg(p.z + row_first + g4 * 4 + lis / (LPR / 4)) : 0.0f;
+        gate[g4] = (EXTRAS && p.z && y_writer) ? __ldg(p.z + row_first + g4 * 4 + lis / (LPR / 4)) : 0.0f;
     const float a = exp_spec(__fmul_rn(dtv, __ldg(p.A + h)));
     const float Dl = (p.D && lis == 0) ? __ldg(p.D + h) : 0.0f;     // the skip term enters the dot on one lane
 
@@ -410,7 +435,8 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
         for (int u = 0; u < 4; ++u) {
             const int k = g4 * 4 + u;
             float hv[EPL];
-            unpack_lane<FMT>(raw[k], hv);
+            cp_async_wait_rows<RPS>(k);                       // rows 0..k have landed
+            unpack_lane<FMT>(tile[k][threadIdx.x], hv);
             const float dtx = __fmul_rn(dtv, xv[k]);
             float dot = __fmul_rn(Dl, xv[k]);
             float amax = 0.0f;
@@ -444,7 +470,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
             if constexpr (RULE == RULE_SR) grp_row += N / 4;
         }
         const float tot = reduce4_over_slot<LPR>(dots[0], dots[1], dots[2], dots[3], lis);
-        if (y_writer) p.y[row_first + g4 * 4 + lis / (LPR / 4)] = p.z ? __fmul_rn(tot, silu(gate[g4])) : tot;
+        if (y_writer) p.y[row_first + g4 * 4 + lis / (LPR / 4)] = (EXTRAS && p.z) ? __fmul_rn(tot, silu(gate[g4])) : tot;
     }
 }
 
@@ -457,12 +483,16 @@ inline cudaError_t launch_update_one(const UpdateParams& p, cudaStream_t stream)
         // shapes the tile kernel covers: a head of nslot * {4, 8} rows; x, y (and row scales) 16-byte aligned
         const bool aligned = ((reinterpret_cast<uintptr_t>(q.x) | reinterpret_cast<uintptr_t>(q.y)) & 15u) == 0 &&
                              (!Fmt<FMT>::kScaled || (reinterpret_cast<uintptr_t>(q.scales) & 15u) == 0);
-        if (aligned && q.P == nslot * 8u) {
-            ssd_update_tile_kernel<FMT, RULE, LPR, 8><<<q.n_items, kThreads, 0, stream>>>(q);
+        const dim3 tile_grid(q.H, q.B);
+        const bool extras = q.dt_bias || q.dt_softplus || q.z || q.ngroups > 1;
+        if (aligned && q.B <= 65535u && q.P == nslot * 8u) {
+            if (extras) ssd_update_tile_kernel<FMT, RULE, LPR, 8, true><<<tile_grid, kThreads, 0, stream>>>(q);
+            else ssd_update_tile_kernel<FMT, RULE, LPR, 8, false><<<tile_grid, kThreads, 0, stream>>>(q);
             return cudaGetLastError();
         }
-        if (aligned && q.P == nslot * 4u) {
-            ssd_update_tile_kernel<FMT, RULE, LPR, 4><<<q.n_items, kThreads, 0, stream>>>(q);
+        if (aligned && q.B <= 65535u && q.P == nslot * 4u) {
+            if (extras) ssd_update_tile_kernel<FMT, RULE, LPR, 4, true><<<tile_grid, kThreads, 0, stream>>>(q);
+            else ssd_update_tile_kernel<FMT, RULE, LPR, 4, false><<<tile_grid, kThreads, 0, stream>>>(q);
             return cudaGetLastError();
         }
     }
