@@ -32,10 +32,9 @@ RULE_IDS = {"rtn": 0, "sr": 1, "weyl": 2, "sr_hash": 3}
 NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the fused update kernel, from the ncu
 # captures summarised under profiles/ (same kernel and per-layer shape as the benchmark's launches).
-NCU_TRAFFIC_BYTES = {(5, "weyl"): 272_856_320 + 214_808_576, (5, "rtn"): 272_839_168 + 213_272_832,
-                     (3, "weyl"): 85_308_416 + 27_165_440, (3, "rtn"): 85_309_184 + 27_241_472,
-                     (4, "weyl"): 17_896_448, (4, "rtn"): 17_885_696}
-FALLBACK_HBM_GBS = 6650.0
+NCU_TRAFFIC_BYTES = {(5, "weyl"): 273_016_576 + 216_289_280, (5, "rtn"): 272_986_368 + 215_508_736,
+                     (3, "weyl"): 85_312_512 + 26_826_496, (3, "rtn"): 85_310_720 + 28_849_664,
+                     (4, "weyl"): 17_895_936, (4, "rtn"): 17_885_696}
 
 
 def measured_peak():
