@@ -389,3 +389,47 @@ def test_checkpointed_rounding(fmt, rule):
     torch.cuda.synchronize()
     assert np.array_equal(codes_to_host(s3, fmt).reshape(-1, N), codes)
     assert np.array_equal(work.cpu().numpy().view(np.uint32), w_h)
+
+
+def test_drivers_carry_the_gate_and_the_options():
+    """z, dt_bias, softplus and groups through ssd_decode_run and ssd_decode_run_host equal per-step calls."""
+    from dataclasses import replace
+    cfg = replace(workloads.CONFIGS[5], batch=2, nheads=4, n_layers=1)
+    B, H, P, N = cfg.state_shape
+    G, T = 2, 6
+    rng = np.random.default_rng(17)
+    f32 = np.float32
+    A, D = workloads.layer_params(cfg)
+    bias = rng.normal(-2, 0.5, H).astype(f32)
+    xs_h = torch.from_numpy(rng.standard_normal((T, 1, B, H, P)).astype(f32)).pin_memory()
+    dts_h = torch.from_numpy(rng.normal(-1, 1, (T, 1, B, H)).astype(f32)).pin_memory()
+    Bs_h = torch.from_numpy((rng.standard_normal((T, 1, B, G, N)) * 0.2).astype(f32)).pin_memory()
+    Cs_h = torch.from_numpy(rng.standard_normal((T, 1, B, G, N)).astype(f32)).pin_memory()
+    zs_h = torch.from_numpy(rng.standard_normal((T, 1, B, H, P)).astype(f32)).pin_memory()
+    xs, dts, Bs, Cs, zs = (t.cuda() for t in (xs_h, dts_h, Bs_h, Cs_h, zs_h))
+
+    def fresh():
+        st = torch.zeros(cfg.state_shape, dtype=torch.int16, device="cuda")
+        return st, ssdq.make_desc(st, None, cfg.fmt, A=to_dev(A), D=to_dev(D), rule=ssdq.WEYL, weyl=ssdq.weyl_offsets_init(0, 0, N),
+                                  dt_bias=to_dev(bias), dt_softplus=True, ngroups=G)
+
+    s1, d1 = fresh()
+    y1 = torch.zeros_like(xs)
+    for t in range(T):
+        ssdq.ssd_state_update(d1, t + 1, x=xs[t, 0], dt=dts[t, 0], Bm=Bs[t, 0], Cm=Cs[t, 0], y=y1[t, 0], z=zs[t, 0])
+    s2, d2 = fresh()
+    y2 = torch.zeros_like(xs)
+    ssdq.ssd_decode_run([d2], 1, T, ssdq.make_step_inputs(xs, dts, Bs, Cs, y2, zs))
+    s3, d3 = fresh()
+    y3_h = torch.zeros_like(xs_h).pin_memory()
+    stg = [torch.zeros((2,) + tuple(t.shape[1:]), dtype=torch.float32, device="cuda") for t in (xs_h, dts_h, Bs_h, Cs_h, y3_h, zs_h)]
+    ssdq.ssd_decode_run_host([d3], 1, T, ssdq.make_step_inputs(xs_h, dts_h, Bs_h, Cs_h, y3_h, zs_h), ssdq.make_step_inputs(*stg))
+    torch.cuda.synchronize()
+    assert torch.equal(s1, s2) and torch.equal(s1, s3)
+    assert torch.equal(y1, y2) and torch.equal(y1.cpu(), y3_h)
+    # and the oracle agrees with the state
+    st, _ = oracle.new_state(cfg.state_shape, cfg.fmt)
+    for t in range(T):
+        oracle.state_update(st, None, cfg.fmt, 0, xs_h[t, 0].numpy(), dts_h[t, 0].numpy(), A, Bs_h[t, 0].numpy(), Cs_h[t, 0].numpy(), D,
+                            oracle.WEYL, t + 1, weyl_block=N, dt_bias=bias, dt_softplus=True, ngroups=G, z=zs_h[t, 0].numpy())
+    assert np.array_equal(codes_to_host(s1, cfg.fmt), st)
