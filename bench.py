@@ -218,8 +218,25 @@ def sweep_batch(args, cfg):
                 sps = args.steps / secs
                 if sps > row.get(name, {}).get("steps_per_s", 0.0):
                     row[name] = {"steps_per_s": sps, "gbs": c.algorithmic_bytes_per_layer_step() * c.n_layers * sps / 1e9}
+        # the same loop replayed as a CUDA graph (write index in device memory): what launch latency costs at small batch
+        stack.set_rule(RULE_IDS["weyl"])
+        counter = torch.zeros(1, dtype=torch.int32, device="cuda")
+        spl = args.ring * max(1, 40 // args.ring)
+        graph = ssdq.DecodeGraph(stack.descs, spl, sin, counter)
+        graph.launch()
+        torch.cuda.synchronize()
+        reps = max(1, args.steps // spl)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            graph.launch()
+        e1.record()
+        e1.synchronize()
+        sps = reps * spl / (e0.elapsed_time(e1) / 1e3)
+        row["weyl_graph"] = {"steps_per_s": sps, "gbs": c.algorithmic_bytes_per_layer_step() * c.n_layers * sps / 1e9}
+        graph.close()
         rows.append(row)
-        del stack, xs, dts, Bs, Cs, sin
+        del stack, xs, dts, Bs, Cs, sin, graph
         torch.cuda.empty_cache()
     print(json.dumps({"metric": "decode_steps_per_s_vs_batch", "config": cfg.name, "layers": cfg.n_layers, "rows": rows}))
 

@@ -165,6 +165,21 @@ typedef struct {
 int ssd_decode_run(const ssdq_update_desc* layers, uint32_t n_layers, uint32_t t_first, uint32_t n_steps,
                    const ssdq_step_inputs* in, void* stream);
 
+/* Replayable CUDA graph of the decode loop, for decode at small batch where the per-layer launches are bound by launch
+ * latency.  ssd_decode_graph_create captures `steps_per_launch` decode steps (steps_per_launch * n_layers fused update
+ * launches, inputs of step i from ring slot i % in->ring; steps_per_launch must be a multiple of in->ring) into a graph
+ * whose kernels read their write index from DEVICE memory: step i of a launch writes with index *step_counter + 1 + i, and
+ * a last node adds steps_per_launch to *step_counter.  The caller owns the counter word (set it to the number of writes
+ * done so far, 0 for a fresh state) and every buffer the descriptors name; all must outlive the graph.
+ * ssd_decode_graph_launch enqueues one replay on `stream`; the caller refreshes the input ring between replays.
+ * The results equal those of ssd_decode_run for the same write indices.  Creation allocates driver-side graph objects
+ * (no device memory of the library's own). */
+typedef struct ssdq_graph ssdq_graph;
+int ssd_decode_graph_create(ssdq_graph** out, const ssdq_update_desc* layers, uint32_t n_layers, uint32_t steps_per_launch,
+                            const ssdq_step_inputs* in, uint32_t* step_counter);
+int ssd_decode_graph_launch(ssdq_graph* graph, void* stream);
+int ssd_decode_graph_destroy(ssdq_graph* graph);
+
 /* Periodic checkpointing (Section 6.5 "Periodic checkpointing"; Appendix B "Decode regime", CC = 8): the state lives in
  * full precision between checkpoints and only every `every`-th write, counted from t_first, is rounded into the store.
  * work_fp32[l] is a caller-owned DEVICE buffer [B, H, P, N] of floats holding layer l's working state (on entry: the

@@ -469,6 +469,92 @@ int ssd_decode_run_host(const ssdq_update_desc* layers, uint32_t n_layers, uint3
     return SSDQ_OK;
 }
 
+struct ssdq_graph {
+    cudaGraph_t graph = nullptr;
+    cudaGraphExec_t exec = nullptr;
+    uint32_t steps = 0, n_layers = 0;
+};
+
+int ssd_decode_graph_create(ssdq_graph** out, const ssdq_update_desc* layers, uint32_t n_layers, uint32_t steps_per_launch,
+                            const ssdq_step_inputs* in, uint32_t* step_counter) {
+    if (!out || !layers || !in || !step_counter) return fail(SSDQ_ERR_NULL, "out, layers, in and step_counter are required");
+    *out = nullptr;
+    if (n_layers == 0 || in->ring == 0 || steps_per_launch == 0) return fail(SSDQ_ERR_SHAPE, "n_layers, ring and steps_per_launch must be positive");
+    if (steps_per_launch % in->ring != 0) return fail(SSDQ_ERR_SHAPE, "steps_per_launch must be a multiple of the input ring");
+    if (!aligned4(step_counter)) return fail(SSDQ_ERR_ALIGN, "step_counter is misaligned");
+    for (uint32_t l = 0; l < n_layers; ++l) {
+        const int rc = check_layer(&layers[l]);
+        if (rc != SSDQ_OK) return rc;
+    }
+    for (uint32_t sl = 0; sl < in->ring; ++sl)
+        for (uint32_t l = 0; l < n_layers; ++l) {
+            const uint64_t k = (uint64_t)sl * n_layers + l;
+            const int rc = check_step_ptrs(in->x + k * in->stride_x, in->dt + k * in->stride_dt, in->Bm + k * in->stride_B,
+                                           in->Cm + k * in->stride_C, in->y + k * in->stride_y, in->z ? in->z + k * in->stride_z : nullptr);
+            if (rc != SSDQ_OK) return rc;
+        }
+    cudaStream_t cs = nullptr;
+    cudaError_t e = cudaStreamCreateWithFlags(&cs, cudaStreamNonBlocking);
+    if (e != cudaSuccess) return fail(SSDQ_ERR_CUDA, "cudaStreamCreate: %s", cudaGetErrorString(e));
+    ssdq_graph* g = new ssdq_graph();
+    g->steps = steps_per_launch;
+    g->n_layers = n_layers;
+    int rc = SSDQ_OK;
+    e = cudaStreamBeginCapture(cs, cudaStreamCaptureModeThreadLocal);
+    if (e != cudaSuccess) rc = fail(SSDQ_ERR_CUDA, "cudaStreamBeginCapture: %s", cudaGetErrorString(e));
+    if (rc == SSDQ_OK) {
+        for (uint32_t i = 0; i < steps_per_launch && rc == SSDQ_OK; ++i)
+            for (uint32_t l = 0; l < n_layers && rc == SSDQ_OK; ++l) {
+                const uint64_t k = (uint64_t)(i % in->ring) * n_layers + l;
+                ssdq::UpdateParams p = make_params(&layers[l], 1u + i);     // write index = counter + 1 + i
+                p.step_base = step_counter;
+                p.x = in->x + k * in->stride_x;
+                p.dt = in->dt + k * in->stride_dt;
+                p.Bm = in->Bm + k * in->stride_B;
+                p.Cm = in->Cm + k * in->stride_C;
+                p.y = in->y + k * in->stride_y;
+                p.z = in->z ? in->z + k * in->stride_z : nullptr;
+                const cudaError_t le = launch_update(p, layers[l].format, layers[l].rule, layers[l].a_per_state != 0, cs);
+                if (le != cudaSuccess) rc = fail(SSDQ_ERR_CUDA, "state-update kernel (capture): %s", cudaGetErrorString(le));
+            }
+        if (rc == SSDQ_OK) {
+            const cudaError_t le = ssdq::launch_counter_add(step_counter, steps_per_launch, cs);
+            if (le != cudaSuccess) rc = fail(SSDQ_ERR_CUDA, "counter kernel (capture): %s", cudaGetErrorString(le));
+        }
+        e = cudaStreamEndCapture(cs, &g->graph);         // always end the capture, also after a failed launch
+        if (rc == SSDQ_OK && e != cudaSuccess) rc = fail(SSDQ_ERR_CUDA, "cudaStreamEndCapture: %s", cudaGetErrorString(e));
+    }
+    if (rc == SSDQ_OK) {
+        e = cudaGraphInstantiate(&g->exec, g->graph, 0);
+        if (e != cudaSuccess) rc = fail(SSDQ_ERR_CUDA, "cudaGraphInstantiate: %s", cudaGetErrorString(e));
+    }
+    cudaStreamDestroy(cs);
+    if (rc != SSDQ_OK) {
+        if (g->exec) cudaGraphExecDestroy(g->exec);
+        if (g->graph) cudaGraphDestroy(g->graph);
+        delete g;
+        return rc;
+    }
+    *out = g;
+    return SSDQ_OK;
+}
+
+int ssd_decode_graph_launch(ssdq_graph* g, void* stream) {
+    if (!g || !g->exec) return fail(SSDQ_ERR_NULL, "graph handle is NULL");
+    const cudaError_t e = cudaGraphLaunch(g->exec, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return fail(SSDQ_ERR_CUDA, "cudaGraphLaunch: %s", cudaGetErrorString(e));
+    g_launches.fetch_add((uint64_t)g->steps * g->n_layers + 1u, std::memory_order_relaxed);
+    return SSDQ_OK;
+}
+
+int ssd_decode_graph_destroy(ssdq_graph* g) {
+    if (!g) return SSDQ_OK;
+    if (g->exec) cudaGraphExecDestroy(g->exec);
+    if (g->graph) cudaGraphDestroy(g->graph);
+    delete g;
+    return SSDQ_OK;
+}
+
 const char* ssdq_last_error(void) { return g_err; }
 
 uint64_t ssdq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

@@ -27,6 +27,7 @@ struct UpdateParams {
     uint32_t scale_block;    // scaled stores: 16 or N
     float scale_top;         // scaled stores: block scale = amax / scale_top (448 for E4M3, q_max for INTb)
     uint32_t step_t;
+    const uint32_t* step_base;   // null, or a device word added to step_t (replayable graphs keep their step count there)
     uint32_t layer;
     uint32_t batch_base;
     uint32_t spi;            // slots per (b, h) item inside a CTA (power of two)
@@ -74,6 +75,7 @@ cudaError_t launch_state_error(const void* codes, const float* scales, const flo
 int report_failure(int status, const char* text);
 void count_launches(unsigned n);
 
+cudaError_t launch_counter_add(uint32_t* counter, uint32_t n, cudaStream_t s);
 cudaError_t launch_readout_kl(const float* y_ref, const float* y_q, uint32_t batch, uint32_t width, float* kl, cudaStream_t s);
 
 }  // namespace ssdq

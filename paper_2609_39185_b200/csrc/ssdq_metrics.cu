@@ -124,6 +124,12 @@ __global__ void __launch_bounds__(kMetricThreads) readout_kl_kernel(const float*
     if (threadIdx.x == 0) kl[blockIdx.x] = (float)acc;
 }
 
+__global__ void counter_add_kernel(uint32_t* counter, uint32_t n) { *counter += n; }
+cudaError_t launch_counter_add(uint32_t* counter, uint32_t n, cudaStream_t s) {
+    counter_add_kernel<<<1, 1, 0, s>>>(counter, n);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_readout_kl(const float* y_ref, const float* y_q, uint32_t batch, uint32_t width, float* kl, cudaStream_t s) {
     readout_kl_kernel<<<batch, kMetricThreads, 0, s>>>(y_ref, y_q, width, kl);
     return cudaGetLastError();

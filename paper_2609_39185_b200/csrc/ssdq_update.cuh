@@ -179,6 +179,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_kernel(const UpdateParams
     constexpr int UNR = Unroll<FMT>::value;
     constexpr unsigned FULL = 0xFFFFFFFFu;
 
+    const uint32_t step_t = p.step_t + (p.step_base ? __ldg(p.step_base) : 0u);
     const uint32_t tid = threadIdx.x;
     const uint32_t lis = tid % LPR;                 // lane in slot
     const uint32_t slot = tid / LPR;
@@ -223,10 +224,10 @@ __global__ void __launch_bounds__(kThreads) ssd_update_kernel(const UpdateParams
     }
 
     LaneThreshold<FMT, RULE, LPR> thr;
-    thr.init(p.weyl, p.step_t, lis);
+    thr.init(p.weyl, step_t, lis);
     const uint32_t key0 = (uint32_t)p.sr_seed, key1 = (uint32_t)(p.sr_seed >> 32);
 
-    const uint32_t hash_base = p.step_t * kHashP2 + p.layer * kHashP3 + key0 * kHashP4;
+    const uint32_t hash_base = step_t * kHashP2 + p.layer * kHashP3 + key0 * kHashP4;
     const uint32_t p_first = sub * p.rps;                         // first row of this slot inside the item
     const uint64_t row_first = (uint64_t)item * p.P + p_first;    // local row index (this call's tensors)
     const uint64_t grow_first = row_first + (uint64_t)p.batch_base * p.H * p.P;   // global row index
@@ -294,7 +295,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_kernel(const UpdateParams
             if constexpr (RULE == RULE_WEYL) acc0 = thr.weyl_acc0(grow_first + k);
             if constexpr (RULE == RULE_SR_HASH) acc0 = thr.hash_key0(grow_first + k, hash_base, key1);
             if constexpr (RULE == RULE_SR) thr.sr_group(grow_first + k, g_lo, g_hi);
-            const uint4 packed = round_pack_lane<FMT, RULE>(hv, acc0, p.weyl.mul_col, g_lo, g_hi, p.step_t, p.layer,
+            const uint4 packed = round_pack_lane<FMT, RULE>(hv, acc0, p.weyl.mul_col, g_lo, g_hi, step_t, p.layer,
                                                              key0, key1, p.scale_top);
             if (ok[u]) state[row * LPR + lis] = packed;
             // y: lane (k mod LPR) of the slot keeps row k; flushed every LPR rows
@@ -360,6 +361,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
     constexpr unsigned FULL = 0xFFFFFFFFu;
     static_assert(RPS % 4 == 0, "rows are processed four at a time");
 
+    const uint32_t step_t = p.step_t + (p.step_base ? __ldg(p.step_base) : 0u);
     const uint32_t lis = threadIdx.x % LPR;
     const uint32_t slot = threadIdx.x / LPR;
     const uint32_t h = blockIdx.x;                  // grid = (H, B): no index division
@@ -419,12 +421,12 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
     const float Dl = (p.D && lis == 0) ? __ldg(p.D + h) : 0.0f;     // the skip term enters the dot on one lane
 
     LaneThreshold<FMT, RULE, LPR> thr;
-    thr.init(p.weyl, p.step_t, lis);
+    thr.init(p.weyl, step_t, lis);
     const uint32_t key0 = (uint32_t)p.sr_seed, key1 = (uint32_t)(p.sr_seed >> 32);
     const uint64_t grow_first = row_first + (uint64_t)p.batch_base * p.H * (NSLOT * RPS);
     uint32_t acc_row = 0;
     uint64_t grp_row = 0;
-    const uint32_t hash_base = p.step_t * kHashP2 + p.layer * kHashP3 + key0 * kHashP4;
+    const uint32_t hash_base = step_t * kHashP2 + p.layer * kHashP3 + key0 * kHashP4;
     if constexpr (RULE == RULE_WEYL) acc_row = thr.weyl_acc0(grow_first);
     if constexpr (RULE == RULE_SR) grp_row = (grow_first * (uint64_t)N + n0) >> 2;
 
@@ -464,7 +466,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
             }
             if constexpr (RULE == RULE_SR_HASH) acc_row = thr.hash_key0(grow_first + k, hash_base, key1);
             const uint4 packed = round_pack_lane<FMT, RULE>(hv, acc_row, p.weyl.mul_col, (uint32_t)grp_row,
-                                                             (uint32_t)(grp_row >> 32), p.step_t, p.layer, key0, key1, p.scale_top);
+                                                             (uint32_t)(grp_row >> 32), step_t, p.layer, key0, key1, p.scale_top);
             sp[k * LPR] = packed;
             if constexpr (RULE == RULE_WEYL) acc_row += thr.row_mul;
             if constexpr (RULE == RULE_SR) grp_row += N / 4;

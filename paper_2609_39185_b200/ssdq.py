@@ -18,7 +18,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libssdq.so")
 
 EXPORTS = ("weyl_offsets_init", "ssdq_thresholds_materialize", "ssd_state_update", "quantize_store",
-           "ssdq_dequantize", "ssd_decode_run", "ssd_decode_run_host", "ssd_replay_step", "ssd_decode_run_checkpointed", "ssdq_state_error_workspace_bytes", "ssdq_state_error",
+           "ssdq_dequantize", "ssd_decode_run", "ssd_decode_run_host", "ssd_replay_step", "ssd_decode_run_checkpointed",
+           "ssd_decode_graph_create", "ssd_decode_graph_launch", "ssd_decode_graph_destroy", "ssdq_state_error_workspace_bytes", "ssdq_state_error",
            "ssdq_state_error_static", "ssdq_readout_kl", "ssdq_last_error", "ssdq_launch_count")
 
 _u32, _u64, _i32, _vp = ctypes.c_uint32, ctypes.c_uint64, ctypes.c_int32, ctypes.c_void_p
@@ -80,6 +81,12 @@ def lib() -> ctypes.CDLL:
         L.ssd_decode_run_checkpointed.restype = ctypes.c_int
         L.ssd_decode_run_checkpointed.argtypes = [ctypes.POINTER(UpdateDesc), ctypes.POINTER(_vp), _u32, _u32, _u32, _u32,
                                                   ctypes.POINTER(StepInputs), _vp]
+        L.ssd_decode_graph_create.restype = ctypes.c_int
+        L.ssd_decode_graph_create.argtypes = [ctypes.POINTER(_vp), ctypes.POINTER(UpdateDesc), _u32, _u32, ctypes.POINTER(StepInputs), _vp]
+        L.ssd_decode_graph_launch.restype = ctypes.c_int
+        L.ssd_decode_graph_launch.argtypes = [_vp, _vp]
+        L.ssd_decode_graph_destroy.restype = ctypes.c_int
+        L.ssd_decode_graph_destroy.argtypes = [_vp]
         L.ssd_decode_run_host.restype = ctypes.c_int
         L.ssd_decode_run_host.argtypes = [ctypes.POINTER(UpdateDesc), _u32, _u32, _u32, ctypes.POINTER(StepInputs),
                                           ctypes.POINTER(StepInputs), _vp]
@@ -256,6 +263,32 @@ def ssd_decode_run_checkpointed(layer_descs, work_states, every: int, t_first: i
     ptrs = (_vp * len(work_states))(*[w.data_ptr() for w in work_states])
     _check(lib().ssd_decode_run_checkpointed(arr, ptrs, len(layer_descs), every, t_first & 0xFFFFFFFF, n_steps,
                                              ctypes.byref(step_inputs), _stream()))
+
+
+class DecodeGraph:
+    """A replayable CUDA graph of `steps_per_launch` decode steps over all layers (ssd_decode_graph_*).  The write index
+    lives in `step_counter`, a CUDA int32 tensor of one element that each replay advances by steps_per_launch."""
+
+    def __init__(self, layer_descs, steps_per_launch: int, step_inputs: StepInputs, step_counter):
+        self._keep = (layer_descs, step_inputs, step_counter)
+        arr = (UpdateDesc * len(layer_descs))(*layer_descs)
+        self.handle = _vp()
+        _check(lib().ssd_decode_graph_create(ctypes.byref(self.handle), arr, len(layer_descs), steps_per_launch,
+                                             ctypes.byref(step_inputs), _ptr(step_counter)))
+
+    def launch(self):
+        _check(lib().ssd_decode_graph_launch(self.handle, _stream()))
+
+    def close(self):
+        if self.handle:
+            lib().ssd_decode_graph_destroy(self.handle)
+            self.handle = _vp()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 def launch_count() -> int:

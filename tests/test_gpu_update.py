@@ -433,3 +433,37 @@ def test_drivers_carry_the_gate_and_the_options():
         oracle.state_update(st, None, cfg.fmt, 0, xs_h[t, 0].numpy(), dts_h[t, 0].numpy(), A, Bs_h[t, 0].numpy(), Cs_h[t, 0].numpy(), D,
                             oracle.WEYL, t + 1, weyl_block=N, dt_bias=bias, dt_softplus=True, ngroups=G, z=zs_h[t, 0].numpy())
     assert np.array_equal(codes_to_host(s1, cfg.fmt), st)
+
+
+@pytest.mark.parametrize("rule", RULES)
+def test_graph_replay_equals_the_plain_driver(rule):
+    """A captured graph of 4 steps x 2 layers, replayed three times with the write index kept in device memory,
+    equals 12 steps of ssd_decode_run."""
+    cfg = workloads.CONFIGS[1].with_batch(3)
+    L, ring, spl, reps = 2, 2, 4, 3
+    params = [workloads.layer_params(cfg, l, l) for l in range(L)]
+    ins = [[workloads.step_inputs(cfg, t + 1, l, l) for l in range(L)] for t in range(ring)]
+    stack = lambda i: to_dev(np.stack([np.stack([ins[t][l][i] for l in range(L)]) for t in range(ring)]))
+    xs, dts, Bs, Cs = (stack(i) for i in range(4))
+
+    def fresh():
+        states = [torch.zeros(cfg.state_shape, dtype=torch.int16, device="cuda") for _ in range(L)]
+        descs = [ssdq.make_desc(states[l], None, cfg.fmt, A=to_dev(params[l][0]), D=to_dev(params[l][1]), rule=rule,
+                                weyl=ssdq.weyl_offsets_init(l, 0, cfg.weyl_block), sr_seed=l, layer=l) for l in range(L)]
+        return states, descs
+
+    s1, d1 = fresh()
+    y1 = torch.zeros_like(xs)
+    ssdq.ssd_decode_run(d1, 1, spl * reps, ssdq.make_step_inputs(xs, dts, Bs, Cs, y1))
+    s2, d2 = fresh()
+    y2 = torch.zeros_like(xs)
+    counter = torch.zeros(1, dtype=torch.int32, device="cuda")
+    graph = ssdq.DecodeGraph(d2, spl, ssdq.make_step_inputs(xs, dts, Bs, Cs, y2), counter)
+    for _ in range(reps):
+        graph.launch()
+    torch.cuda.synchronize()
+    assert int(counter.item()) == spl * reps
+    for l in range(L):
+        assert torch.equal(s1[l], s2[l])
+    assert torch.equal(y1, y2)
+    graph.close()
