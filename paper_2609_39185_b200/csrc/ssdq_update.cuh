@@ -336,6 +336,7 @@ __device__ __forceinline__ float reduce4_over_slot(float d0, float d1, float d2,
 // cp.async.wait_group needs an immediate: allow at most RPS - 1 - k groups (the rows after k) to be pending.
 template <int RPS>
 __device__ __forceinline__ void cp_async_wait_rows(int k) {
+    static_assert(RPS <= 16, "one commit group per row, at most 16 rows per lane");
     switch (RPS - 1 - k) {
         case 0: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;
         case 1: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
@@ -344,14 +345,36 @@ __device__ __forceinline__ void cp_async_wait_rows(int k) {
         case 4: asm volatile("cp.async.wait_group 4;" ::: "memory"); break;
         case 5: asm volatile("cp.async.wait_group 5;" ::: "memory"); break;
         case 6: asm volatile("cp.async.wait_group 6;" ::: "memory"); break;
-        default: asm volatile("cp.async.wait_group 7;" ::: "memory"); break;
+        case 7: asm volatile("cp.async.wait_group 7;" ::: "memory"); break;
+        case 8: asm volatile("cp.async.wait_group 8;" ::: "memory"); break;
+        case 9: asm volatile("cp.async.wait_group 9;" ::: "memory"); break;
+        case 10: asm volatile("cp.async.wait_group 10;" ::: "memory"); break;
+        case 11: asm volatile("cp.async.wait_group 11;" ::: "memory"); break;
+        case 12: asm volatile("cp.async.wait_group 12;" ::: "memory"); break;
+        case 13: asm volatile("cp.async.wait_group 13;" ::: "memory"); break;
+        case 14: asm volatile("cp.async.wait_group 14;" ::: "memory"); break;
+        default: asm volatile("cp.async.wait_group 15;" ::: "memory"); break;
     }
+}
+
+// The same for two rows (slots of at least two lanes): returns the total of row j = lane_in_slot / (LPR / 2).
+template <int LPR>
+__device__ __forceinline__ float reduce2_over_slot(float d0, float d1, uint32_t lis) {
+    static_assert(LPR >= 2, "needs at least two lanes per row");
+    constexpr unsigned FULL = 0xFFFFFFFFu;
+    const bool hi = (lis & (LPR / 2)) != 0;
+    float k = hi ? d1 : d0;
+    const float s = hi ? d0 : d1;
+    k += __shfl_xor_sync(FULL, s, LPR / 2);
+#pragma unroll
+    for (int off = LPR / 4; off > 0; off >>= 1) k += __shfl_xor_sync(FULL, k, off);
+    return k;
 }
 
 // The tile kernel: the same computation for the shapes that dominate (one decay per head, a head of
 // P = (kThreads / LPR) * RPS rows), one CTA per (b, h).  A head's state is one contiguous tile (16 KB for
-// 64 x 128 two-byte codes); every lane issues all RPS of its 128-bit state loads, the x row and its
-// constants before touching any of them, then walks its rows four at a time.  No guards, no idle lanes.
+// 64 x 128 two-byte codes), staged through shared memory; rows are walked GRP = min(4, RPS) at a time so that their
+// readout dots share one transposed reduction.  No guards, no idle lanes.
 // EXTRAS: any of dt_bias, in-kernel softplus, B/C groups or the z gate is in use (the plain step pays nothing for them).
 template <int FMT, int RULE, int LPR, int RPS, bool EXTRAS>
 __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateParams p) {
@@ -359,7 +382,8 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
     constexpr int N = LPR * EPL;
     constexpr int NSLOT = kThreads / LPR;
     constexpr unsigned FULL = 0xFFFFFFFFu;
-    static_assert(RPS % 4 == 0, "rows are processed four at a time");
+    constexpr int GRP = RPS >= 4 ? 4 : 2;        // rows per reduction group
+    static_assert(RPS % GRP == 0 && LPR >= GRP, "rows are processed GRP at a time by slots of at least GRP lanes");
 
     const uint32_t step_t = p.step_t + (p.step_base ? __ldg(p.step_base) : 0u);
     const uint32_t lis = threadIdx.x % LPR;
@@ -386,9 +410,14 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
     float xv[RPS];
     float sc[Fmt<FMT>::kScaled ? RPS : 1];
 #pragma unroll
-    for (int k = 0; k < RPS / 4; ++k) {
-        const float4 x4 = __ldg(reinterpret_cast<const float4*>(p.x + row_first) + k);
-        xv[4 * k] = x4.x; xv[4 * k + 1] = x4.y; xv[4 * k + 2] = x4.z; xv[4 * k + 3] = x4.w;
+    for (int k = 0; k < RPS / GRP; ++k) {
+        if constexpr (GRP == 4) {
+            const float4 x4 = __ldg(reinterpret_cast<const float4*>(p.x + row_first) + k);
+            xv[4 * k] = x4.x; xv[4 * k + 1] = x4.y; xv[4 * k + 2] = x4.z; xv[4 * k + 3] = x4.w;
+        } else {
+            const float2 x2 = __ldg(reinterpret_cast<const float2*>(p.x + row_first) + k);
+            xv[2 * k] = x2.x; xv[2 * k + 1] = x2.y;
+        }
     }
     if constexpr (Fmt<FMT>::kScaled) {
 #pragma unroll
@@ -411,12 +440,12 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
         if (p.dt_bias) dtv = __fadd_rn(dtv, __ldg(p.dt_bias + h));
         if (p.dt_softplus) dtv = softplus_spec(dtv);
     }
-    // the lanes that will write y fetch their gate values now (row j = lane_in_slot / (LPR / 4) of each group of four)
-    const bool y_writer = (lis & (LPR / 4 - 1)) == 0;
-    float gate[RPS / 4];
+    // the lanes that will write y fetch their gate values now (row j = lane_in_slot / (LPR / GRP) of each group)
+    const bool y_writer = (lis & (LPR / GRP - 1)) == 0;
+    float gate[RPS / GRP];
 #pragma unroll
-    for (int g4 = 0; g4 < RPS / 4; ++g4)
-        gate[g4] = (EXTRAS && p.z && y_writer) ? __ldg(p.z + row_first + g4 * 4 + lis / (LPR / 4)) : 0.0f;
+    for (int g4 = 0; g4 < RPS / GRP; ++g4)
+        gate[g4] = (EXTRAS && p.z && y_writer) ? __ldg(p.z + row_first + g4 * GRP + lis / (LPR / GRP)) : 0.0f;
     const float a = exp_spec(__fmul_rn(dtv, __ldg(p.A + h)));
     const float Dl = (p.D && lis == 0) ? __ldg(p.D + h) : 0.0f;     // the skip term enters the dot on one lane
 
@@ -431,11 +460,11 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
     if constexpr (RULE == RULE_SR) grp_row = (grow_first * (uint64_t)N + n0) >> 2;
 
 #pragma unroll
-    for (int g4 = 0; g4 < RPS / 4; ++g4) {
-        float dots[4];
+    for (int g4 = 0; g4 < RPS / GRP; ++g4) {
+        float dots[GRP];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int k = g4 * 4 + u;
+        for (int u = 0; u < GRP; ++u) {
+            const int k = g4 * GRP + u;
             float hv[EPL];
             cp_async_wait_rows<RPS>(k);                       // rows 0..k have landed
             unpack_lane<FMT>(tile[k][threadIdx.x], hv);
@@ -471,8 +500,10 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
             if constexpr (RULE == RULE_WEYL) acc_row += thr.row_mul;
             if constexpr (RULE == RULE_SR) grp_row += N / 4;
         }
-        const float tot = reduce4_over_slot<LPR>(dots[0], dots[1], dots[2], dots[3], lis);
-        if (y_writer) p.y[row_first + g4 * 4 + lis / (LPR / 4)] = (EXTRAS && p.z) ? __fmul_rn(tot, silu(gate[g4])) : tot;
+        float tot;
+        if constexpr (GRP == 4) tot = reduce4_over_slot<LPR>(dots[0], dots[1], dots[2], dots[3], lis);
+        else tot = reduce2_over_slot<LPR>(dots[0], dots[1], lis);
+        if (y_writer) p.y[row_first + g4 * GRP + lis / (LPR / GRP)] = (EXTRAS && p.z) ? __fmul_rn(tot, silu(gate[g4])) : tot;
     }
 }
 
@@ -482,20 +513,23 @@ inline cudaError_t launch_update_one(const UpdateParams& p, cudaStream_t stream)
     UpdateParams q = p;
     const uint32_t nslot = kThreads / LPR;
     if constexpr (!APS && LPR >= 4 && FMT != FMT_FP32) {
-        // shapes the tile kernel covers: a head of nslot * {4, 8} rows; x, y (and row scales) 16-byte aligned
+        // shapes the tile kernel covers: a head of nslot * {2, 4, 8, 16} rows; x, y (and row scales) 16-byte aligned
         const bool aligned = ((reinterpret_cast<uintptr_t>(q.x) | reinterpret_cast<uintptr_t>(q.y)) & 15u) == 0 &&
                              (!Fmt<FMT>::kScaled || (reinterpret_cast<uintptr_t>(q.scales) & 15u) == 0);
         const dim3 tile_grid(q.H, q.B);
         const bool extras = q.dt_bias || q.dt_softplus || q.z || q.ngroups > 1;
-        if (aligned && q.B <= 65535u && q.P == nslot * 8u) {
-            if (extras) ssd_update_tile_kernel<FMT, RULE, LPR, 8, true><<<tile_grid, kThreads, 0, stream>>>(q);
-            else ssd_update_tile_kernel<FMT, RULE, LPR, 8, false><<<tile_grid, kThreads, 0, stream>>>(q);
-            return cudaGetLastError();
-        }
-        if (aligned && q.B <= 65535u && q.P == nslot * 4u) {
-            if (extras) ssd_update_tile_kernel<FMT, RULE, LPR, 4, true><<<tile_grid, kThreads, 0, stream>>>(q);
-            else ssd_update_tile_kernel<FMT, RULE, LPR, 4, false><<<tile_grid, kThreads, 0, stream>>>(q);
-            return cudaGetLastError();
+        if (aligned && q.B <= 65535u) {
+#define SSDQ_TILE_CASE(R)                                                                                          \
+            if (q.P == nslot * (R)) {                                                                              \
+                if (extras) ssd_update_tile_kernel<FMT, RULE, LPR, R, true><<<tile_grid, kThreads, 0, stream>>>(q);  \
+                else ssd_update_tile_kernel<FMT, RULE, LPR, R, false><<<tile_grid, kThreads, 0, stream>>>(q);       \
+                return cudaGetLastError();                                                                         \
+            }
+            SSDQ_TILE_CASE(8u)
+            SSDQ_TILE_CASE(4u)
+            if constexpr (Fmt<FMT>::kBytes == 2) { SSDQ_TILE_CASE(16u) }     // P = 128 or N = 256 with two-byte codes
+            if constexpr (Fmt<FMT>::kBytes == 1) { SSDQ_TILE_CASE(2u) }      // small heads with one-byte codes
+#undef SSDQ_TILE_CASE
         }
     }
     uint32_t spi = 1;

@@ -106,6 +106,8 @@ SHAPES = [
     # (B, H, P, N, a_per_state)
     (1, 1, 1, 16, False), (3, 5, 7, 16, True), (2, 3, 64, 128, False), (5, 7, 3, 128, False), (2, 2, 100, 64, False),
     (1, 9, 8, 256, False), (2, 130, 1, 32, True), (1, 3, 65, 128, True), (4, 1, 16, 64, True),
+    # heads the tile kernel takes with 16, 2 and 4 rows per slot
+    (2, 3, 128, 128, False), (1, 2, 64, 256, False), (2, 3, 32, 128, False), (2, 2, 64, 64, False), (2, 2, 32, 64, False),
 ]
 
 
