@@ -89,30 +89,40 @@ __device__ __forceinline__ uint4 round_pack_lane(const float* v, uint32_t acc0, 
             }
         }
         if constexpr (FMT == FMT_BF16) {
-            uint32_t any = 0;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                w[i] = trunc_pack2_bf16(dither_sum_bf16(v[2 * i], acc[2 * i]), dither_sum_bf16(v[2 * i + 1], acc[2 * i + 1]));
-                any |= w[i];
-            }
-            if (any & 0x40004000u) {   // some |code| >= 2: it may sit at the top of the range, take the clamped route
-#pragma unroll
-                for (int i = 0; i < 4; ++i)
-                    w[i] = dither_code_bf16_clamped(v[2 * i], acc[2 * i]) | (dither_code_bf16_clamped(v[2 * i + 1], acc[2 * i + 1]) << 16);
+                const uint32_t b0 = __float_as_uint(v[2 * i]), b1 = __float_as_uint(v[2 * i + 1]);
+                const uint32_t x0 = acc[2 * i] ^ (uint32_t)((int32_t)b0 >> 31);        // a negative value takes ~U
+                const uint32_t x1 = acc[2 * i + 1] ^ (uint32_t)((int32_t)b1 >> 31);
+                w[i] = sr_pack2_bf16(v[2 * i], v[2 * i + 1], x0, x1);
             }
         } else if constexpr (FMT == FMT_FP16) {
+            uint32_t unsure = 0;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                float r[2];
+                const uint32_t b0 = __float_as_uint(v[2 * i]), b1 = __float_as_uint(v[2 * i + 1]);
+                const uint32_t x0 = acc[2 * i] ^ (uint32_t)((int32_t)b0 >> 31);
+                const uint32_t x1 = acc[2 * i + 1] ^ (uint32_t)((int32_t)b1 >> 31);
+                const uint32_t f = (x0 >> 19) | ((x1 >> 3) & 0x1FFF0000u);              // the leading 13 bits of each
+                const uint32_t f1 = f + 0x00010001u;
+                w[i] = sr_pack2_fp16(v[2 * i], v[2 * i + 1], f);
+                // the true addend lies in [f, f + 1): if the next field gives another code, or does not fit, decide exactly
+                unsure |= (w[i] ^ sr_pack2_fp16(v[2 * i], v[2 * i + 1], f1)) | (f1 & 0x20002000u);
+            }
+            if (unsure) {
 #pragma unroll
-                for (int j = 0; j < 2; ++j) {
-                    const float vv = v[2 * i + j];
-                    const float scale = dither_step_scale<10, -14, 24>(vv);
-                    const float q = floor_to_step(dithered_sum_rm(vv, acc[2 * i + j], scale), scale);
-                    // sign of v forced onto the result (it already has it unless it is zero)
-                    r[j] = __uint_as_float((__float_as_uint(q) & 0x7FFFFFFFu) | (__float_as_uint(vv) & 0x80000000u));
+                for (int i = 0; i < 4; ++i) {
+                    float r[2];
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        const float vv = v[2 * i + j];
+                        const float scale = dither_step_scale<10, -14, 24>(vv);
+                        const float q = floor_to_step(dithered_sum_rm(vv, acc[2 * i + j], scale), scale);
+                        // sign of v forced onto the result (it already has it unless it is zero)
+                        r[j] = __uint_as_float((__float_as_uint(q) & 0x7FFFFFFFu) | (__float_as_uint(vv) & 0x80000000u));
+                    }
+                    w[i] = rtn_pack2_fp16(r[0], r[1]);   // exact: r is on the FP16 grid; saturates beyond 65504
                 }
-                w[i] = rtn_pack2_fp16(r[0], r[1]);   // exact: r is on the FP16 grid; saturates beyond 65504
             }
         } else if constexpr (FMT == FMT_INT) {
 #pragma unroll
