@@ -57,7 +57,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantParams p)
                 for (int off = LPR / 2; off > 0; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, off));
             }
             const float s = fmaxf(__fdiv_rn(amax, p.scale_top), 1.17549435e-38f);
-            const float rinv = __fdiv_rn(1.0f, s);
+            const float rinv = __frcp_rn(s);
 #pragma unroll
             for (int j = 0; j < EPL; ++j) v[j] = __fmul_rn(v[j], rinv);
             if (ok) {
