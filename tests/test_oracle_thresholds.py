@@ -210,3 +210,31 @@ def test_hash_sr_definition_and_moments():
     vals = [star_discrepancy([oracle.threshold(oracle.SR_HASH, flat=2000 + j, t=t) / 2.0**24 for t in range(1, 257)])
             for j in range(200)]
     assert abs(np.mean(vals) - 0.0539) < 0.004
+
+
+def test_discrepancy_utility_reproduces_table_8_for_other_increments():
+    """The star-discrepancy utility used by the pins above, checked on sequences the oracle does not implement:
+    LD_256 of Weyl dithers with other increments (Table 8), float64 phase reduced modulo 1."""
+    phi = (1 + math.sqrt(5)) / 2
+    rows = {"sqrt2-1": (math.sqrt(2) - 1, 0.0069), "1/(2+phi)": (1 / (2 + phi), 0.0075), "e-2": (math.e - 2, 0.0097),
+            "1/4+2^-12": (0.25 + 2.0**-12, 0.1379), "1/3+2^-12": (1 / 3 + 2.0**-12, 0.2063), "1/2+2^-12": (0.5 + 2.0**-12, 0.3347)}
+    rng = np.random.default_rng(12)
+    for name, (alpha, want) in rows.items():
+        vals = []
+        for _ in range(400):      # more starts than the paper's 64: the near-rational rows vary strongly with the offset
+            o, t0 = rng.random(), int(rng.integers(1, 1 << 20))
+            u = (o + (np.arange(t0, t0 + 256) * alpha) % 1.0) % 1.0
+            vals.append(star_discrepancy(u))
+        assert abs(np.mean(vals) - want) < max(0.0008, 0.06 * want), name
+
+
+def test_near_rational_increment_is_as_bad_as_rtn():
+    # Corollary 1(d): alpha = 1/2 + eps leaves two empty arcs of length 3/8 for T <= 1/(8 eps): D*_T >= 3/16
+    eps = 2.0**-12
+    T = int(1 / (8 * eps))
+    for o in (0.0, 0.3, 0.77):
+        u = (o + np.arange(1, T + 1) * (0.5 + eps)) % 1.0
+        assert star_discrepancy(u) >= 3 / 16 - 1e-9
+    # while the golden-ratio sequence of the same length is two orders of magnitude more even
+    u = np.array([oracle.weyl_u24(NO_OFFSET, NO_OFFSET, 0, 0, t) for t in range(1, T + 1)]) / 2.0**24
+    assert star_discrepancy(u) < 0.01
