@@ -182,3 +182,42 @@ def test_dithers_are_unbiased_and_lemma_2_noise(rule):
     assert abs(np.mean(res**2) - 1 / 6) < 0.004
     res = (oracle.round_values(xs, 0, FP16, RTN).astype(np.float64) - xs.astype(np.float64)) / s
     assert abs(np.mean(res**2) - 1 / 12) < 0.002
+
+
+@pytest.mark.parametrize("fmt,lo,hi", [(FP16, -60, 18), (BF16, -126, 127), (E4M3, -40, 10)])
+def test_dithered_rounding_on_a_million_values(fmt, lo, hi):
+    """The case form of Eq. 2 on the enumerated grid, vectorised in float64 (every quantity below is exact in
+    float64: grid points and values are binary32 numbers, the spacing is a power of two, u is a multiple of 2^-24)."""
+    rng = np.random.default_rng(30 + fmt)
+    grid = grid_of(fmt)
+    n = 1_000_000
+    v = sample_values(rng, n, lo, hi)
+    v[::1000] = 0.0
+    v = v[np.abs(v) <= MAX_FINITE[fmt]]
+    U = rng.integers(0, 1 << 24, len(v)).astype(np.uint32)
+    U[::9] = 0
+    U[1::9] = (1 << 24) - 1
+    vd = v.astype(np.float64)
+    i = np.searchsorted(grid, vd, side="right") - 1
+    lo_pt = grid[i]
+    hi_pt = grid[np.minimum(i + 1, len(grid) - 1)]
+    on_grid = lo_pt == vd
+    step = np.where(on_grid, 1.0, hi_pt - lo_pt)
+    f = (vd - lo_pt) / step
+    up = (U.astype(np.float64) / 2.0**24 >= 1.0 - f) & ~on_grid
+    want = np.where(up, hi_pt, lo_pt)
+    got = oracle.round_values(v, U, fmt, WEYL).astype(np.float64)
+    assert np.array_equal(got, want)
+    zero = got == 0.0
+    assert np.array_equal(np.signbit(got[zero]), np.signbit(v[zero]))
+
+
+@pytest.mark.parametrize("fmt", [FP16, BF16, E4M3])
+def test_rtn_matches_native_casts_on_two_million_values(fmt):
+    rng = np.random.default_rng(40 + fmt)
+    lo, hi = {FP16: (-60, 16), BF16: (-126, 127), E4M3: (-40, 9)}[fmt]
+    v = sample_values(rng, 2_000_000, lo, hi)
+    v = v[np.abs(v) <= MAX_FINITE[fmt]]
+    want = torch.from_numpy(v).to(TORCH_DTYPE[fmt]).to(torch.float32).numpy()
+    got = oracle.round_values(v, 0, fmt, RTN)
+    assert np.array_equal(want.view(np.uint32), got.view(np.uint32))
