@@ -102,6 +102,7 @@ ssdq::UpdateParams make_params(const ssdq_update_desc* d, uint32_t step_t) {
     p.n_items = d->batch * d->nheads;
     p.scale_block = d->scale_block;
     p.scale_top = scale_top(d->format);
+    p.inv_scale_top = 1.0f / p.scale_top;
     p.step_t = step_t; p.layer = d->layer; p.batch_base = d->batch_index_base;
     p.weyl = weyl_const(d->weyl);
     p.sr_seed = d->sr_seed;

@@ -26,6 +26,7 @@ struct UpdateParams {
     uint32_t n_items;        // B * H
     uint32_t scale_block;    // scaled stores: 16 or N
     float scale_top;         // scaled stores: block scale = amax / scale_top (448 for E4M3, q_max for INTb)
+    float inv_scale_top;     // RN(1 / scale_top)
     uint32_t step_t;
     const uint32_t* step_base;   // null, or a device word added to step_t (replayable graphs keep their step count there)
     uint32_t layer;

@@ -1,0 +1,453 @@
+// ssdq_stream.cuh -- the fused decode step as a persistent, software-pipelined kernel for the block-scaled
+// one-byte stores (E4M3 and INTb with FP32 scales), where the work per byte moved is largest.
+//
+// Why a second kernel.  With one-byte codes a head's tile is only 8 KB and a CTA spends most of its life
+// computing, so a kernel that loads its tile, computes and exits keeps too few bytes in flight to fill HBM
+// (it ran at half the copy bandwidth with the issue slots half idle).  Here a CTA stays resident and walks a
+// contiguous range of (b, h) items; the codes, x and scales of the next STAGES - 1 items are already on their way
+// (cp.async into a ring of shared-memory stages, one commit group per item) while the current one is computed,
+// so the memory system always has several tiles per CTA outstanding.  Each lane reads back only what it copied
+// itself: cp.async.wait_group is the only synchronisation, there is no barrier and no wait on another thread.
+//
+// Arithmetic.  The same operations in the same order as ssd_update_tile_kernel (every stored bit is identical),
+// issued two entries at a time with the packed binary32 instructions of sm_100 (mul/fma/add .f32x2, all rounding
+// modes), the three-input max for the block maximum, a division by the format's constant that is exact by
+// construction, and -- for the E4M3 dither -- Eq. 2 in integer form on the binary32 bits.
+#pragma once
+#include "ssdq_update.cuh"
+
+#ifndef SSDQ_STREAM_MINB
+#define SSDQ_STREAM_MINB 5
+#endif
+
+namespace ssdq {
+
+// ---- two binary32 values in one 64-bit register pair ------------------------------------------------------------
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) { f32x2 r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi)); return r; }
+__device__ __forceinline__ f32x2 pack2u(uint32_t lo, uint32_t hi) { f32x2 r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi)); return r; }
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ void unpack2u(f32x2 v, uint32_t& lo, uint32_t& hi) { asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v)); }
+__device__ __forceinline__ f32x2 mul2_rn(f32x2 a, f32x2 b) { f32x2 r; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+__device__ __forceinline__ f32x2 add2_rn(f32x2 a, f32x2 b) { f32x2 r; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+__device__ __forceinline__ f32x2 add2_rm(f32x2 a, f32x2 b) { f32x2 r; asm("add.rm.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+__device__ __forceinline__ f32x2 fma2_rn(f32x2 a, f32x2 b, f32x2 c) { f32x2 r; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c)); return r; }
+__device__ __forceinline__ f32x2 fma2_rm(f32x2 a, f32x2 b, f32x2 c) { f32x2 r; asm("fma.rm.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c)); return r; }
+// max(m, |a|, |b|) and min(m, |a|, |b|) in one instruction
+__device__ __forceinline__ float max3abs(float m, float a, float b) { float r; asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(m), "f"(fabsf(a)), "f"(fabsf(b))); return r; }
+__device__ __forceinline__ float min3abs(float m, float a, float b) { float r; asm("min.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(m), "f"(fabsf(a)), "f"(fabsf(b))); return r; }
+
+// amax / top, correctly rounded, for the constant tops of the scaled stores (448, 127, 63, 31, 7): with c = RN(1/top),
+// q = RN(amax c), r = amax - top q (exact in one fma) and RN(q + r c) is the correctly rounded quotient -- checked
+// against IEEE division for every binary32 significand and each of the five constants.  A small amax is scaled by
+// 2^64 first so that no intermediate underflows; scaling back rounds only when the quotient is below the smallest
+// normal number, where the caller's floor at that number hides it.  Only for max(result, FLT_MIN).
+__device__ __forceinline__ float div_by_top(float amax, float top, float inv_top) {
+    const bool small = amax < 0x1p-60f;
+    const float a = __fmul_rn(amax, small ? 0x1p64f : 1.0f);
+    const float q = __fmul_rn(a, inv_top);
+    const float r = __fmaf_rn(__fmaf_rn(-top, q, a), inv_top, q);
+    return __fmul_rn(r, small ? 0x1p-64f : 1.0f);
+}
+
+// Unpack one 32-bit word of one-byte codes into two packed pairs (exact widening).
+__device__ __forceinline__ void unpack4_e4m3_x2(uint32_t w, f32x2& p01, f32x2& p23) {
+    float f[4];
+    unpack4_e4m3(w, f);
+    p01 = pack2(f[0], f[1]);
+    p23 = pack2(f[2], f[3]);
+}
+__device__ __forceinline__ void unpack4_int8_x2(uint32_t w, f32x2& p01, f32x2& p23) {
+    w ^= 0x80808080u;                                      // bias to unsigned bytes
+    const f32x2 off = pack2(-8388736.0f, -8388736.0f);     // -(2^23 + 128)
+    p01 = add2_rn(pack2u(__byte_perm(w, 0x4B000000u, 0x7540), __byte_perm(w, 0x4B000000u, 0x7541)), off);
+    p23 = add2_rn(pack2u(__byte_perm(w, 0x4B000000u, 0x7542), __byte_perm(w, 0x4B000000u, 0x7543)), off);
+}
+
+// ---- rounding of a lane's 16 scaled values (8 packed pairs) into 16 one-byte codes ------------------------------
+// four binary32 values -> four E4M3 codes in memory order (v0 in the low byte), round to nearest even, saturating
+__device__ __forceinline__ uint32_t rtn_pack4_e4m3(float v0, float v1, float v2, float v3) {
+    uint32_t r;
+    asm("{.reg .b16 lo, hi; cvt.rn.satfinite.e4m3x2.f32 lo, %2, %1; cvt.rn.satfinite.e4m3x2.f32 hi, %4, %3; mov.b32 %0, {lo, hi};}"
+        : "=r"(r) : "f"(v0), "f"(v1), "f"(v2), "f"(v3));
+    return r;
+}
+// The stochastic-rounding convert with all random bits zero adds nothing and truncates the magnitude onto the E4M3
+// grid (subnormal targets and saturation included: compared with the exact convert of the truncated value on every
+// binary32 pattern).  Its first operand lands in the HIGH byte.
+__device__ __forceinline__ uint32_t trunc_pack4_e4m3(float v0, float v1, float v2, float v3) {
+    uint32_t r;
+    asm("cvt.rs.satfinite.e4m3x4.f32 %0, {%1, %2, %3, %4}, %5;" : "=r"(r) : "f"(v3), "f"(v2), "f"(v1), "f"(v0), "r"(0u));
+    return r;
+}
+
+// acc[k]: the threshold word of entry k (U = acc >> 8); unused under RTN.
+template <int FMT, int RULE>
+__device__ __forceinline__ uint4 round_pack_lane_x2(const f32x2* v2, const uint32_t* acc, float qmax, float vmin) {
+    uint32_t w[4];
+    if constexpr (RULE == RULE_RTN) {
+        if constexpr (FMT == FMT_E4M3) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                float a, b, c, d;
+                unpack2(v2[2 * i], a, b);
+                unpack2(v2[2 * i + 1], c, d);
+                w[i] = rtn_pack4_e4m3(a, b, c, d);
+            }
+        } else {
+            const f32x2 magic = pack2(kIntMagic, kIntMagic);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                uint32_t t0, t1, t2, t3;
+                unpack2u(add2_rn(v2[2 * i], magic), t0, t1);         // nearest-even integer in the low mantissa bits
+                unpack2u(add2_rn(v2[2 * i + 1], magic), t2, t3);
+                w[i] = pack4_low_bytes(t0, t1, t2, t3);
+            }
+        }
+    } else if constexpr (FMT == FMT_INT) {
+        // clamp(floor(v + u)): the sum rounded down, then the add of the magic floors it (Eq. 2 on the integer grid);
+        // the integers sit in the low halves of the sums, where they are clamped two at a time
+        const f32x2 magic = pack2(kIntMagic, kIntMagic), ulp = pack2(0x1p-32f, 0x1p-32f);
+        const uint32_t q = (uint32_t)(int)qmax, hi2 = q | (q << 16), lo2 = (uint32_t)(-(int)q & 0xFFFF) * 0x00010001u;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            uint32_t kk[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int k = 4 * i + 2 * h;
+                const f32x2 u2 = pack2(__uint2float_rn(acc[k] & 0xFFFFFF00u), __uint2float_rn(acc[k + 1] & 0xFFFFFF00u));   // exact: 24 bits
+                uint32_t t0, t1;
+                unpack2u(add2_rm(fma2_rm(u2, ulp, v2[k / 2]), magic), t0, t1);
+                kk[h] = __vimax3_s16x2(__vimin3_s16x2(__byte_perm(t0, t1, 0x5410), hi2, hi2), lo2, lo2);
+            }
+            w[i] = __byte_perm(kk[0], kk[1], 0x6420);
+        }
+    } else {
+        // E4M3 dither.  Every |v| >= 2^-6 has an E4M3 target in the normal range: 20 binary32 mantissa bits are
+        // dropped, and floor(v / 2^q + u) adds the leading 20 bits of (threshold XOR sign mask) to the sign-magnitude
+        // bits and truncates; the carry crosses binades by itself and the convert saturates.  A lane with a smaller
+        // value (zero included) takes Eq. 2 literally in binary32 instead.
+        if (vmin >= 0x1p-6f) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                float r[4];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t b0, b1;
+                    unpack2u(v2[2 * i + h], b0, b1);
+                    const int k = 4 * i + 2 * h;
+                    const uint32_t x0 = acc[k] ^ (uint32_t)((int32_t)b0 >> 31), x1 = acc[k + 1] ^ (uint32_t)((int32_t)b1 >> 31);
+                    r[2 * h] = __uint_as_float(b0 + (x0 >> 12));
+                    r[2 * h + 1] = __uint_as_float(b1 + (x1 >> 12));
+                }
+                w[i] = trunc_pack4_e4m3(r[0], r[1], r[2], r[3]);
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                float r[4], vv[4];
+                unpack2(v2[2 * i], vv[0], vv[1]);
+                unpack2(v2[2 * i + 1], vv[2], vv[3]);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float scale = dither_step_scale<3, -6, 127>(vv[j]);
+                    const float q = floor_to_step(dithered_sum_rm(vv[j], acc[4 * i + j], scale), scale);
+                    r[j] = __uint_as_float((__float_as_uint(q) & 0x7FFFFFFFu) | (__float_as_uint(vv[j]) & 0x80000000u));
+                }
+                w[i] = rtn_pack4_e4m3(r[0], r[1], r[2], r[3]);   // exact; saturates beyond 448
+            }
+        }
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async16_ca(uint32_t smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async4_ca(uint32_t smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int PENDING>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory"); }
+
+// Shared memory of one CTA: STAGES x { codes [RPS][kThreads] x 16 B, x [RPS/4][kThreads] x 16 B, scales [RPS/4][kThreads] x 16 B }.
+template <int RPS, int STAGES>
+constexpr size_t stream_smem_bytes() { return (size_t)STAGES * kThreads * 16u * (RPS + 2 * (RPS / 4)); }
+
+// One-byte block-scaled stores, one decay per head, heads of P = (kThreads / LPR) * RPS rows, RPS a multiple of 4.
+// ROW_SCALE: one scale per row of N entries (else one per 16 entries = per lane).
+// grid = any number of CTAs <= n_items; CTA c owns items [c n / G, (c + 1) n / G).
+template <int FMT, int RULE, int LPR, int RPS, int STAGES, bool ROW_SCALE>
+__global__ void __launch_bounds__(kThreads, SSDQ_STREAM_MINB) ssd_update_stream_kernel(const UpdateParams p) {
+    static_assert(Fmt<FMT>::kScaled && Fmt<FMT>::kEpl == 16, "one-byte block-scaled stores");
+    static_assert(RPS % 4 == 0 && LPR >= 4 && STAGES >= 2, "rows are processed four at a time");
+    constexpr int EPL = 16;
+    constexpr int N = LPR * EPL;
+    constexpr int NSLOT = kThreads / LPR;
+    constexpr int ROWS = NSLOT * RPS;
+    constexpr int SPR = ROW_SCALE ? 1 : N / 16;            // scales per row
+    constexpr unsigned FULL = 0xFFFFFFFFu;
+    constexpr uint32_t kTileStage = RPS * kThreads * 16u, kVecStage = (RPS / 4) * kThreads * 16u;
+
+    extern __shared__ uint4 stream_smem[];
+    const uint32_t tid = threadIdx.x;
+    const uint32_t lis = tid % LPR;
+    const uint32_t slot = tid / LPR;
+    const uint32_t n0 = lis * EPL;
+    // this lane's cell of every stage: byte addresses in the shared window
+    const uint32_t tile_s = (uint32_t)__cvta_generic_to_shared(stream_smem) + tid * 16u;    // + stage * kTileStage + k * kThreads * 16
+    const uint32_t x_s = tile_s + STAGES * kTileStage;                                       // + stage * kVecStage + k4 * kThreads * 16
+    const uint32_t sc_s = x_s + STAGES * kVecStage;
+
+    const uint32_t first = (uint32_t)(((uint64_t)blockIdx.x * p.n_items) / gridDim.x);
+    const uint32_t last = (uint32_t)(((uint64_t)(blockIdx.x + 1) * p.n_items) / gridDim.x);
+    if (first >= last) return;
+    const uint32_t step_t = p.step_t + (p.step_base ? __ldg(p.step_base) : 0u);
+    const float top = p.scale_top, inv_top = p.inv_scale_top;
+
+    // pointers of the item being fetched (f_*) and of the item being computed (c_*), advanced by one item per iteration
+    const uint64_t row0 = (uint64_t)first * ROWS + slot * RPS;
+    const uint4* f_codes = reinterpret_cast<const uint4*>(p.state) + row0 * LPR + lis;
+    const float* f_x = p.x + row0;
+    const float* f_sc = p.scales + row0 * SPR + (ROW_SCALE ? 0u : lis);
+    uint4* c_codes = reinterpret_cast<uint4*>(p.state) + row0 * LPR + lis;
+    float* c_sc = p.scales + row0 * SPR + (ROW_SCALE ? 0u : lis);
+    float* c_y = p.y + row0 + lis / (LPR / 4);
+
+    auto issue = [&](uint32_t stage) {
+#pragma unroll
+        for (int k = 0; k < RPS; ++k) cp_async16(tile_s + stage * kTileStage + k * (kThreads * 16u), f_codes + k * LPR);
+#pragma unroll
+        for (int k4 = 0; k4 < RPS / 4; ++k4) {
+            cp_async16_ca(x_s + stage * kVecStage + k4 * (kThreads * 16u), f_x + 4 * k4);
+            const uint32_t sdst = sc_s + stage * kVecStage + k4 * (kThreads * 16u);
+            if constexpr (ROW_SCALE) {
+                cp_async16_ca(sdst, f_sc + 4 * k4);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) cp_async4_ca(sdst + 4 * j, f_sc + (4 * k4 + j) * SPR);
+            }
+        }
+        f_codes += ROWS * LPR;
+        f_x += ROWS;
+        f_sc += ROWS * SPR;
+    };
+#pragma unroll
+    for (int s = 0; s < STAGES - 1; ++s) {
+        if (first + s < last) issue(s);
+        cp_async_commit();
+    }
+
+    LaneThreshold<FMT, RULE, LPR> thr;
+    thr.init(p.weyl, step_t, lis);
+    const uint32_t key0 = (uint32_t)p.sr_seed, key1 = (uint32_t)(p.sr_seed >> 32);
+    const uint32_t hash_base = step_t * kHashP2 + p.layer * kHashP3 + key0 * kHashP4;
+    const bool y_writer = (lis & (LPR / 4 - 1)) == 0;
+    uint64_t grow_first = row0 + (uint64_t)p.batch_base * p.H * ROWS;
+
+    uint32_t b = first / p.H;
+    uint32_t h = first - b * p.H;
+    f32x2 B2[EPL / 2], C2[EPL / 2];
+    // scalars of the next item are fetched one iteration ahead
+    float dt_next = __ldg(p.dt + first), A_next = __ldg(p.A + h), D_next = (p.D && lis == 0) ? __ldg(p.D + h) : 0.0f;
+
+    uint32_t stage = 0;
+    uint32_t item = first;
+    while (item < last) {
+      // a run of items of one sequence b shares B and C
+      {
+        const float4* Bp = reinterpret_cast<const float4*>(p.Bm + (size_t)b * N + n0);
+        const float4* Cp = reinterpret_cast<const float4*>(p.Cm + (size_t)b * N + n0);
+#pragma unroll
+        for (int i = 0; i < EPL / 4; ++i) {
+            const float4 bb = __ldg(Bp + i), cc = __ldg(Cp + i);
+            B2[2 * i] = pack2(bb.x, bb.y); B2[2 * i + 1] = pack2(bb.z, bb.w);
+            C2[2 * i] = pack2(cc.x, cc.y); C2[2 * i + 1] = pack2(cc.z, cc.w);
+        }
+      }
+      const uint32_t run_end = min(last, (b + 1u) * p.H);
+      for (; item < run_end; ++item) {
+        // refill the stage that the previous iteration consumed
+        {
+            uint32_t fill = stage + (STAGES - 1);
+            if (fill >= STAGES) fill -= STAGES;
+            if (item + (STAGES - 1) < last) issue(fill);
+            cp_async_commit();
+        }
+        const float dtv = dt_next, Dl = D_next;
+        const float a = exp_spec(__fmul_rn(dtv, A_next));
+        if (item + 1 < last) {
+            const uint32_t h_n = (h + 1u == p.H) ? 0u : h + 1u;
+            dt_next = __ldg(p.dt + item + 1);
+            A_next = __ldg(p.A + h_n);
+            D_next = (p.D && lis == 0) ? __ldg(p.D + h_n) : 0.0f;
+        }
+        uint32_t acc_row = 0;
+        uint64_t grp_row = 0;
+        if constexpr (RULE == RULE_WEYL) acc_row = thr.weyl_acc0(grow_first);
+        if constexpr (RULE == RULE_SR) grp_row = (grow_first * (uint64_t)N + n0) >> 2;
+        const f32x2 a2 = pack2(a, a);
+
+        cp_async_wait<STAGES - 1>();                  // this item's group has landed (later ones may be pending)
+        // one row: dequantise, Eq. 1, partial dot, block scale, thresholds, Eq. 2, store; returns the lane's partial dot
+        auto process_row = [&](const int k, const float xk, const float sk) -> float {
+            uint32_t rw[4];
+            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(rw[0]), "=r"(rw[1]), "=r"(rw[2]), "=r"(rw[3]) : "r"(tile_s + stage * kTileStage + k * (kThreads * 16u)));
+            f32x2 hv[EPL / 2];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                if constexpr (FMT == FMT_E4M3) unpack4_e4m3_x2(rw[i], hv[2 * i], hv[2 * i + 1]);
+                else unpack4_int8_x2(rw[i], hv[2 * i], hv[2 * i + 1]);
+            }
+            const float dtx = __fmul_rn(dtv, xk);
+            const f32x2 dtx2 = pack2(dtx, dtx), sc2 = pack2(sk, sk);
+            f32x2 dotA = pack2(__fmul_rn(Dl, xk), 0.0f), dotB = pack2(0.0f, 0.0f);
+            float amaxA = 0.0f, amaxB = 0.0f;
+#pragma unroll
+            for (int i = 0; i < EPL / 2; i += 2) {
+                const f32x2 Bi0 = B2[i], Bi1 = B2[i + 1], Ci0 = C2[i], Ci1 = C2[i + 1];
+                const f32x2 hn0 = fma2_rn(a2, mul2_rn(hv[i], sc2), mul2_rn(dtx2, Bi0));
+                const f32x2 hn1 = fma2_rn(a2, mul2_rn(hv[i + 1], sc2), mul2_rn(dtx2, Bi1));
+                hv[i] = hn0;
+                hv[i + 1] = hn1;
+                dotA = fma2_rn(Ci0, hn0, dotA);
+                dotB = fma2_rn(Ci1, hn1, dotB);
+                float e0, e1, e2, e3;
+                unpack2(hn0, e0, e1);
+                unpack2(hn1, e2, e3);
+                amaxA = max3abs(amaxA, e0, e1);
+                amaxB = max3abs(amaxB, e2, e3);
+            }
+            float d0, d1;
+            unpack2(add2_rn(dotA, dotB), d0, d1);
+            float amax = fmaxf(amaxA, amaxB);
+            if constexpr (ROW_SCALE) {
+#pragma unroll
+                for (int off = LPR / 2; off > 0; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, off));
+            }
+            const float s = fmaxf(div_by_top(amax, top, inv_top), 1.17549435e-38f);
+            const float rinv = __frcp_rn(s);
+            const f32x2 rinv2 = pack2(rinv, rinv);
+            float vminA = 3.0e38f, vminB = 3.0e38f;
+#pragma unroll
+            for (int i = 0; i < EPL / 2; i += 2) {
+                hv[i] = mul2_rn(hv[i], rinv2);
+                hv[i + 1] = mul2_rn(hv[i + 1], rinv2);
+                if constexpr (FMT == FMT_E4M3 && RULE != RULE_RTN) {
+                    float e0, e1, e2, e3;
+                    unpack2(hv[i], e0, e1);
+                    unpack2(hv[i + 1], e2, e3);
+                    vminA = min3abs(vminA, e0, e1);
+                    vminB = min3abs(vminB, e2, e3);
+                }
+            }
+            if constexpr (ROW_SCALE) { if (lis == 0) c_sc[k] = s; }
+            else c_sc[k * SPR] = s;
+
+            uint32_t acc[EPL];
+            if constexpr (RULE == RULE_WEYL) {
+#pragma unroll
+                for (int j = 0; j < EPL; ++j) acc[j] = acc_row + (uint32_t)j * p.weyl.mul_col;
+                acc_row += thr.row_mul;
+            } else if constexpr (RULE == RULE_SR_HASH) {
+                const uint32_t key = thr.hash_key0(grow_first + k, hash_base, key1);
+#pragma unroll
+                for (int j = 0; j < EPL; ++j) acc[j] = fmix32(key + (uint32_t)j * kHashP1);
+            } else if constexpr (RULE == RULE_SR) {
+#pragma unroll
+                for (int g = 0; g < EPL / 4; ++g) {
+                    const uint4 o = philox4x32_10(make_uint4((uint32_t)grp_row + (uint32_t)g, (uint32_t)(grp_row >> 32), step_t, p.layer), key0, key1);
+                    acc[4 * g] = o.x; acc[4 * g + 1] = o.y; acc[4 * g + 2] = o.z; acc[4 * g + 3] = o.w;
+                }
+                grp_row += N / 4;
+            }
+            c_codes[k * LPR] = round_pack_lane_x2<FMT, RULE>(hv, acc, top, fminf(vminA, vminB));
+            return __fadd_rn(d0, d1);
+        };
+#pragma unroll
+        for (int g4 = 0; g4 < RPS / 4; ++g4) {
+            float4 x4, s4;
+            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(x4.x), "=f"(x4.y), "=f"(x4.z), "=f"(x4.w) : "r"(x_s + stage * kVecStage + g4 * (kThreads * 16u)));
+            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(s4.x), "=f"(s4.y), "=f"(s4.z), "=f"(s4.w) : "r"(sc_s + stage * kVecStage + g4 * (kThreads * 16u)));
+            const float d0 = process_row(g4 * 4 + 0, x4.x, s4.x);
+            const float d1 = process_row(g4 * 4 + 1, x4.y, s4.y);
+            const float d2 = process_row(g4 * 4 + 2, x4.z, s4.z);
+            const float d3 = process_row(g4 * 4 + 3, x4.w, s4.w);
+            const float tot = reduce4_over_slot<LPR>(d0, d1, d2, d3, lis);
+            if (y_writer) c_y[g4 * 4] = tot;
+        }
+        c_codes += ROWS * LPR;
+        c_sc += ROWS * SPR;
+        c_y += ROWS;
+        grow_first += ROWS;
+        ++h;
+        if (++stage == STAGES) stage = 0;
+      }
+      h = 0;
+      ++b;
+    }
+    cp_async_wait<0>();
+}
+
+// ---- host side --------------------------------------------------------------------------------------------------
+// Resident CTAs per SM of one instantiation on the current device, and the device's SM count (queried once each).
+template <int FMT, int RULE, int LPR, int RPS, int STAGES, bool ROW_SCALE>
+inline cudaError_t stream_geometry(int& ctas_per_sm, int& sms) {
+    constexpr int kMaxDevices = 64;
+    static int cached_ctas[kMaxDevices] = {}, cached_sms[kMaxDevices] = {};     // per device; a race only repeats the queries
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (cached_ctas[dev] == 0) {
+        auto kernel = ssd_update_stream_kernel<FMT, RULE, LPR, RPS, STAGES, ROW_SCALE>;
+        constexpr size_t smem = stream_smem_bytes<RPS, STAGES>();
+        if ((e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+        int n = 0, occ = 0;
+        if ((e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+        if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kThreads, smem)) != cudaSuccess) return e;
+        if (occ < 1 || n < 1) return cudaErrorInvalidConfiguration;
+        cached_sms[dev] = n;
+        cached_ctas[dev] = occ;
+    }
+    ctas_per_sm = cached_ctas[dev];
+    sms = cached_sms[dev];
+    return cudaSuccess;
+}
+
+template <int FMT, int RULE, int LPR, int RPS, int STAGES, bool ROW_SCALE>
+inline cudaError_t launch_stream(const UpdateParams& p, cudaStream_t stream) {
+    int ctas = 0, sms = 0;
+    const cudaError_t e = stream_geometry<FMT, RULE, LPR, RPS, STAGES, ROW_SCALE>(ctas, sms);
+    if (e != cudaSuccess) return e;
+    uint32_t grid = (uint32_t)(ctas * sms);            // one wave of resident CTAs
+    if (grid > p.n_items) grid = p.n_items;
+    ssd_update_stream_kernel<FMT, RULE, LPR, RPS, STAGES, ROW_SCALE><<<grid, kThreads, stream_smem_bytes<RPS, STAGES>(), stream>>>(p);
+    return cudaGetLastError();
+}
+
+// Shapes covered: N = 128 with heads of 64 or 128 rows, the plain signature (no dt_bias / softplus / groups / gate),
+// x, y and the scales 16-byte aligned.  Two stages: one item in flight per CTA besides the one being computed was
+// the fastest setting measured (more stages cost resident CTAs).
+template <int FMT, int RULE, int LPR>
+cudaError_t try_launch_stream(const UpdateParams& p, cudaStream_t stream, bool& launched) {
+    launched = false;
+    if constexpr (LPR == 8) {
+        const bool extras = p.dt_bias || p.dt_softplus || p.z || p.ngroups > 1;
+        const bool aligned = ((reinterpret_cast<uintptr_t>(p.x) | reinterpret_cast<uintptr_t>(p.y) | reinterpret_cast<uintptr_t>(p.scales)) & 15u) == 0;
+        constexpr uint32_t nslot = kThreads / LPR;
+        if (extras || !aligned || !(p.P == nslot * 4u || p.P == nslot * 8u)) return cudaSuccess;
+        launched = true;
+        const bool row_scale = p.scale_block == (uint32_t)(LPR * 16);
+        if (p.P == nslot * 4u)
+            return row_scale ? launch_stream<FMT, RULE, LPR, 4, 2, true>(p, stream) : launch_stream<FMT, RULE, LPR, 4, 2, false>(p, stream);
+        return row_scale ? launch_stream<FMT, RULE, LPR, 8, 2, true>(p, stream) : launch_stream<FMT, RULE, LPR, 8, 2, false>(p, stream);
+    }
+    return cudaSuccess;
+}
+
+}  // namespace ssdq

@@ -517,11 +517,20 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
     }
 }
 
+// The persistent kernel of ssdq_stream.cuh, for the shapes it covers; `launched` says whether it took the call.
+template <int FMT, int RULE, int LPR>
+cudaError_t try_launch_stream(const UpdateParams& p, cudaStream_t stream, bool& launched);
+
 // Host-side launcher for one (format, rule): picks the lanes-per-row instantiation from N.
 template <int FMT, int RULE, int LPR, bool APS>
 inline cudaError_t launch_update_one(const UpdateParams& p, cudaStream_t stream) {
     UpdateParams q = p;
     const uint32_t nslot = kThreads / LPR;
+    if constexpr (!APS && LPR >= 4 && Fmt<FMT>::kScaled && Fmt<FMT>::kBytes == 1) {
+        bool launched = false;
+        const cudaError_t e = try_launch_stream<FMT, RULE, LPR>(q, stream, launched);
+        if (launched || e != cudaSuccess) return e;
+    }
     if constexpr (!APS && LPR >= 4 && FMT != FMT_FP32) {
         // shapes the tile kernel covers: a head of nslot * {2, 4, 8, 16} rows; x, y (and row scales) 16-byte aligned
         const bool aligned = ((reinterpret_cast<uintptr_t>(q.x) | reinterpret_cast<uintptr_t>(q.y)) & 15u) == 0 &&

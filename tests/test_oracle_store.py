@@ -1,0 +1,158 @@
+"""Pins of the oracle's stand-alone store functions and of its sanity metrics.
+
+quantize_store / replay_step: the dither index of entry (row, col) is the flat index of the [-1, row_len] view
+that starts `row_index_base` rows into the layer's state, flat = (row_index_base + row) * row_len + col, and block r,
+position c of Appendix B "Dithers" are flat / block and flat % block.  Each stored code is rebuilt here element by
+element from the separately pinned pieces (threshold, Eq. 2 on the grid, encode), so a dropped or unscaled base fails.
+
+state_error_per_head / readout_kl: the metric of Appendix B "Open-loop replay" and the KL of Section 4
+"What we measure", on cases small enough to write the answer out by hand.
+"""
+from fractions import Fraction
+import math
+
+import numpy as np
+import pytest
+
+import oracle
+from oracle import FP16, BF16, E4M3, FP32, INT8, INT4, RTN, SR, WEYL, SR_HASH
+
+f32 = np.float32
+TINY = np.finfo(np.float32).tiny
+TOP = {E4M3: 448.0, INT8: 127.0, INT4: 7.0}
+
+# row bases: none, a few rows, and one that carries the flat index past 2^32
+BASES = [0, 5, (1 << 32) // 32 + 7]
+
+
+def _expected_codes(hp, fmt, rule, step_t, base, *, scale_block, weyl_block, layer, weyl_seed, sr_seed):
+    """Codes and scales of the FP32 rows `hp` [n_rows, row_len], one entry at a time."""
+    n_rows, row_len = hp.shape
+    codes = np.zeros(hp.shape, dtype=oracle.CODE_DTYPE[fmt])
+    scaled = oracle.has_block_scale(fmt)
+    scales = np.zeros((n_rows, row_len // scale_block), f32) if scaled else None
+    for row in range(n_rows):
+        for col in range(row_len):
+            v = hp[row, col]
+            if scaled:
+                k0 = (col // scale_block) * scale_block
+                amax = np.max(np.abs(hp[row, k0:k0 + scale_block]))
+                s = max(f32(amax / f32(TOP[fmt])), TINY)
+                scales[row, col // scale_block] = s
+                v = f32(v * f32(f32(1.0) / s))
+            flat = (base + row) * row_len + col
+            U = oracle.threshold(rule, flat, step_t, layer=layer, weyl_seed=weyl_seed, weyl_block=weyl_block, sr_seed=sr_seed)
+            codes[row, col] = oracle.encode(oracle.round_values(v, U, fmt, rule), fmt)[0]
+    return codes, scales
+
+
+@pytest.mark.parametrize("fmt", [FP16, BF16, E4M3, INT8, INT4])
+@pytest.mark.parametrize("rule", [SR, WEYL, SR_HASH])
+@pytest.mark.parametrize("base", BASES)
+def test_quantize_store_dither_index_follows_row_index_base(fmt, rule, base):
+    rng = np.random.default_rng(1000 * fmt + 10 * rule + (base % 7))
+    n_rows, row_len = 6, 32
+    sb = 16 if oracle.has_block_scale(fmt) else 0
+    src = (rng.standard_normal((n_rows, row_len)) * rng.uniform(0.01, 3.0, (n_rows, 1))).astype(f32)
+    kw = dict(scale_block=sb, weyl_block=16, layer=3, weyl_seed=2, sr_seed=0x1234567890)
+    got_c, got_s = oracle.quantize_store(src, fmt, rule, 7, row_index_base=base, **kw)
+    want_c, want_s = _expected_codes(src, fmt, rule, 7, base, **kw)
+    assert np.array_equal(got_c, want_c)
+    if want_s is not None:
+        assert np.array_equal(got_s, want_s)
+    # the base matters: the same rows quantised with another base draw other thresholds
+    other_c, _ = oracle.quantize_store(src, fmt, rule, 7, row_index_base=base + 1, **kw)
+    assert not np.array_equal(other_c, got_c)
+    # ... and it is the ROW count that is added: rows 2.. of a store based at `base` are rows 0.. of one based at base + 2
+    tail_c, _ = oracle.quantize_store(src[2:], fmt, rule, 7, row_index_base=base + 2, **kw)
+    assert np.array_equal(tail_c, got_c[2:])
+
+
+def test_quantize_store_weyl_block_equal_to_the_row():
+    # block = row_len: r is the global row, c the column (the hybrid-shaped configurations)
+    rng = np.random.default_rng(77)
+    src = rng.standard_normal((4, 64)).astype(f32)
+    got, _ = oracle.quantize_store(src, BF16, WEYL, 9, weyl_block=64, layer=1, row_index_base=11)
+    for row in range(4):
+        for col in range(64):
+            U = oracle.weyl_u24(11 + row, col, 1, 0, 9)
+            assert got[row, col] == oracle.encode(oracle.round_values(src[row, col], U, BF16, WEYL), BF16)[0]
+
+
+def _fma32(a, h, w):
+    """One fused multiply-add in binary32: exact product and sum, a single rounding."""
+    return f32(float(Fraction(float(a)) * Fraction(float(h)) + Fraction(float(w))))
+
+
+@pytest.mark.parametrize("fmt", [FP16, BF16, E4M3, INT8])
+@pytest.mark.parametrize("rule", [SR, WEYL, SR_HASH])
+@pytest.mark.parametrize("base", BASES)
+def test_replay_step_dither_index_follows_row_index_base(fmt, rule, base):
+    rng = np.random.default_rng(2000 * fmt + 10 * rule + (base % 7))
+    n_rows, row_len, rpd = 4, 32, 2
+    sb = 16 if oracle.has_block_scale(fmt) else 0
+    kw = dict(scale_block=sb, weyl_block=16, layer=1, weyl_seed=4, sr_seed=99)
+    h0 = rng.standard_normal((n_rows, row_len)).astype(f32)
+    codes, scales = oracle.quantize_store(h0, fmt, RTN, 1, scale_block=sb)
+    w = (0.3 * rng.standard_normal((n_rows, row_len))).astype(f32)
+    a = rng.uniform(0.5, 1.0, n_rows // rpd).astype(f32)
+    h_in = oracle.decode(codes, fmt)
+    if scales is not None:
+        h_in = (h_in.reshape(n_rows, -1, sb) * scales[:, :, None]).astype(f32).reshape(n_rows, row_len)
+    hp = np.array([[_fma32(a[r // rpd], h_in[r, c], w[r, c]) for c in range(row_len)] for r in range(n_rows)], dtype=f32)
+    want_c, want_s = _expected_codes(hp, fmt, rule, 12, base, **kw)
+    got_c = codes.copy()
+    got_s = None if scales is None else scales.copy()
+    oracle.replay_step(w, a, rpd, got_c, got_s, fmt, rule, 12, row_index_base=base, **kw)
+    assert np.array_equal(got_c, want_c)
+    if want_s is not None:
+        assert np.array_equal(got_s, want_s)
+    other = codes.copy()
+    oracle.replay_step(w, a, rpd, other, None if scales is None else scales.copy(), fmt, rule, 12, row_index_base=base + 1, **kw)
+    assert not np.array_equal(other, got_c)
+
+
+# ---- sanity metrics, by hand -----------------------------------------------------------------------
+def test_state_error_per_head_on_a_case_written_out_by_hand():
+    # B = 2, H = 2, P = 1, N = 16, FP16 codes (every value below is an FP16 number).  Head 0: the store equals the
+    # twin except for two entries off by 1/4 and 1/2; head 1: every entry of the store is the twin's plus 1/8.
+    B, H, P, N = 2, 2, 1, 16
+    twin = np.zeros((B, H, P, N), f32)
+    twin[0, 0, 0, :] = 1.0                       # sum of squares 16
+    twin[1, 0, 0, :] = 2.0                       # 64
+    twin[0, 1, 0, :] = 0.5                       # 4
+    twin[1, 1, 0, :] = -1.0                      # 16
+    stored = twin.copy()
+    stored[0, 0, 0, 3] += 0.25                   # 1/16
+    stored[1, 0, 0, 9] -= 0.5                    # 1/4
+    stored[:, 1] += 0.125                        # 32 entries * 1/64 = 1/2
+    codes = oracle.encode(stored, FP16)
+    err2, ref2 = oracle.state_error_per_head(codes, None, twin, FP16)
+    assert err2.tolist() == [1 / 16 + 1 / 4, 0.5]
+    assert ref2.tolist() == [80.0, 20.0]
+    # a scaled store: INT8 codes k with one scale per row, h_hat = k * s
+    k = np.zeros((B, H, P, N), np.int8)
+    k[0, 0, 0, 0], k[1, 1, 0, 5] = 127, -64
+    scales = np.array([0.5, 1.0, 1.0, 0.25], f32)              # rows (b, h) = (0,0), (0,1), (1,0), (1,1)
+    tw = np.zeros((B, H, P, N), f32)
+    tw[0, 0, 0, 0], tw[1, 1, 0, 5] = 63.0, -15.0               # h_hat = 63.5 and -16
+    err2, ref2 = oracle.state_error_per_head(k.view(np.uint8), scales, tw, INT8, 16)
+    assert err2.tolist() == [0.25, 1.0]
+    assert ref2.tolist() == [63.0**2, 225.0]
+
+
+def test_readout_kl_on_a_case_written_out_by_hand():
+    ln2 = math.log(2.0)
+    # sequence 0: p = softmax(0, ln 2) = (1/3, 2/3), q = softmax(0, 0) = (1/2, 1/2)
+    # sequence 1: p = (1/2, 1/4, 1/4), q = (1/4, 1/4, 1/2), given as log-weights with an arbitrary common shift
+    y_ref = np.array([[0.0, ln2, -1e30], [3.0 + ln2, 3.0, 3.0]])
+    y_q = np.array([[7.0, 7.0, -1e30], [-1.0, -1.0, -1.0 + ln2]])
+    got = oracle.readout_kl(y_ref, y_q)
+    want0 = (1 / 3) * math.log((1 / 3) / (1 / 2)) + (2 / 3) * math.log((2 / 3) / (1 / 2))
+    want1 = 0.5 * math.log(2.0) + 0.25 * math.log(1.0) + 0.25 * math.log(0.5)
+    assert got == pytest.approx([want0, want1], rel=1e-12)
+    assert np.all(oracle.readout_kl(y_ref, y_ref) == 0.0)
+    # not symmetric: KL(q || p) is another number
+    assert oracle.readout_kl(y_q, y_ref)[0] == pytest.approx(0.5 * math.log(0.5 / (1 / 3)) + 0.5 * math.log(0.5 / (2 / 3)), rel=1e-12)
+    # shape: any trailing dimensions are flattened per sequence
+    assert oracle.readout_kl(y_ref.reshape(2, 3, 1), y_q.reshape(2, 3, 1)) == pytest.approx([want0, want1], rel=1e-12)
