@@ -30,15 +30,16 @@ from paper_2609_39185_b200 import workloads  # noqa: E402
 
 RULE_IDS = {"rtn": 0, "sr": 1, "weyl": 2, "sr_hash": 3}
 NOMINAL_HBM_GBS = 8000.0
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the fused update kernel, from the ncu
-# captures summarised under profiles/ (same kernel and per-layer shape as the benchmark's launches).
-NCU_TRAFFIC_BYTES = {(5, "weyl"): 273_016_576 + 216_289_280, (5, "rtn"): 272_986_368 + 215_508_736,
-                     (3, "weyl"): 85_312_512 + 26_826_496, (3, "rtn"): 85_310_720 + 28_849_664,
-                     (4, "weyl"): 17_895_936, (4, "rtn"): 17_885_696}
+FALLBACK_HBM_GBS = 6650.0      # an earlier stream-copy measurement on this machine, used only if MEASURED_PEAKS.json is absent
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the fused update kernel from the one-kernel ncu
+# captures summarised under profiles/ (same kernel and per-layer shape as the benchmark's launches; see NCU_TRAFFIC_SOURCE).
+# A launch ends with part of its last writes still in L2, so the write term undercounts by up to the L2 size.
+NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_SOURCE = "profiles/ssd_update_tile_kernel_bf16_config5.md (one launch, 2 layers resident)"
 
 
-def measured_peak():
-    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+def measured_peak(path=None):
+    path = path or os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         try:
             return float(json.load(open(path))["hbm_gbs"]), "measured (MEASURED_PEAKS.json, stream copy)"
@@ -141,48 +142,73 @@ def time_steps(stack, step_inputs, t_first, n_steps):
     return e0.elapsed_time(e1) / 1e3
 
 
+class OracleSample:
+    """The CPU oracle, as it stands, on a bounded sample of the workload: sequences 0..7 of every layer (sequences are
+    independent, so the sample is an exact slice of the full batch)."""
+
+    def __init__(self, cfg, rule, seed=0):
+        import oracle
+        self.oracle, self.cfg, self.rule = oracle, cfg, rule
+        self.nb = min(cfg.batch, 8)
+        self.sub = cfg.with_batch(self.nb)
+        self.layers = []
+        for l in range(cfg.n_layers):
+            ls = workloads.layer_seed(cfg, seed, l)
+            A, D = workloads.layer_params(cfg, l, ls)
+            st, sc = oracle.new_state(self.sub.state_shape, cfg.fmt, cfg.scale_block)
+            self.layers.append((ls, A, D, st, sc))
+        self.ins = {l: workloads.step_inputs(cfg, 1, l, self.layers[l][0], slice(0, self.nb)) for l in range(cfg.n_layers)}
+        oracle.lib()
+        self.t = 0
+
+    def step(self):
+        self.t += 1
+        for l, (ls, A, D, st, sc) in enumerate(self.layers):
+            x, dt, Bm, Cm = self.ins[l]
+            self.oracle.state_update(st, sc, self.cfg.fmt, self.cfg.scale_block, x, dt, A, Bm, Cm, D, self.rule, self.t, layer=l,
+                                     weyl_block=self.cfg.weyl_block, sr_seed=ls)
+
+    def timed(self, steps):
+        t0 = time.perf_counter()
+        for _ in range(steps):
+            self.step()
+        return time.perf_counter() - t0
+
+    def report(self, steps, secs):
+        bytes_per_step = self.sub.algorithmic_bytes_per_layer_step() * self.cfg.n_layers
+        gbs = bytes_per_step * steps / secs / 1e9
+        info = (f"{steps} steps of {self.cfg.n_layers} layers on sequences 0..{self.nb - 1} of {self.cfg.batch} "
+                f"({secs:.1f} s)")
+        return gbs, info
+
+
 def oracle_sample(cfg, rule, seed=0, target_seconds=12.0):
-    """The CPU oracle, as it stands, on a bounded sample of the same workload: a slice of the batch of
-    every layer, decoded for a few steps on the host cores.  Returns (GB/s, steps/s at full batch, info)."""
-    import oracle
-    nb = min(cfg.batch, 8)
-    sub = cfg.with_batch(nb)
-    per_layer = []
-    for l in range(cfg.n_layers):
-        ls = workloads.layer_seed(cfg, seed, l)
-        A, D = workloads.layer_params(cfg, l, ls)
-        st, sc = oracle.new_state(sub.state_shape, cfg.fmt, cfg.scale_block)
-        per_layer.append((ls, A, D, st, sc))
-    ins = {l: workloads.step_inputs(cfg, 1, l, per_layer[l][0], slice(0, nb)) for l in range(cfg.n_layers)}
-    oracle.lib()
-    t0 = time.perf_counter()
-    steps = 0
-    while True:
-        for l, (ls, A, D, st, sc) in enumerate(per_layer):
-            x, dt, Bm, Cm = ins[l]
-            oracle.state_update(st, sc, cfg.fmt, cfg.scale_block, x, dt, A, Bm, Cm, D, rule, steps + 1, layer=l,
-                                weyl_block=cfg.weyl_block, sr_seed=ls)
-        steps += 1
-        el = time.perf_counter() - t0
-        if el > target_seconds or steps >= 64:
-            break
-    bytes_per_step = sub.algorithmic_bytes_per_layer_step() * cfg.n_layers
-    gbs = bytes_per_step * steps / el / 1e9
-    full_steps_per_s = steps / el * nb / cfg.batch
-    info = f"{steps} steps of {cfg.n_layers} layers on sequences 0..{nb - 1} of {cfg.batch} ({el:.1f} s)"
-    return gbs, full_steps_per_s, oracle.num_threads(), info
+    """About target_seconds of oracle work for the cpu_baseline key.  Returns (GB/s, steps/s at full batch, cores, info)."""
+    o = OracleSample(cfg, rule, seed)
+    first = o.timed(1)
+    steps = int(max(2, min(64, target_seconds / max(first, 1e-3))))
+    secs = o.timed(steps)
+    gbs, info = o.report(steps, secs)
+    return gbs, steps / secs * o.nb / cfg.batch, o.oracle.num_threads(), info
 
 
 def run_reference(args, cfg):
+    """The reference arm: W warm-up steps, then exactly K timed steps of the oracle, each step one decode step of the
+    bounded sample (sequences 0..7 of every layer); rank 0 only."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    gbs, sps, cores, info = oracle_sample(cfg, RULE_IDS[args.rule], target_seconds=max(4.0, 3.0 * args.steps))
+    o = OracleSample(cfg, RULE_IDS[args.rule])
+    o.timed(min(args.warmup, 3))
+    secs = o.timed(args.steps)
+    gbs, info = o.report(args.steps, secs)
+    ms_sample = secs / args.steps * 1e3
     line = {"impl": "reference", "metric": "state_update_hbm_gbs", "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 / sps if sps else None,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_sample,
+            "ms_per_step_extrapolated_full_batch": ms_sample * cfg.batch / o.nb,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": workload_config(cfg, args),
-            "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": info},
+            "config": dict(workload_config(cfg, args), sample=f"sequences 0..{o.nb - 1} of {cfg.batch} per step"),
+            "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": o.oracle.num_threads(), "kind": "oracle", "sample": info},
             "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
@@ -196,6 +222,36 @@ def workload_config(cfg, args):
             "l2": "state larger than L2 (no flush needed)" if cfg.state_bytes_per_layer() * cfg.n_layers > 256e6
                   else "state may be L2-resident",
             "parallelism": f"replicas x{args.gpus} (batch shards, no collective)"}
+
+
+def formats_table(cfg, peak, xs, dts, Bs, Cs, layers=2, rounds=7, reps=20):
+    """RTN and Weyl on the configuration's per-layer shape for each store format: algorithmic GB/s, fraction of the measured
+    peak and the Weyl/RTN time ratio (interleaved rounds, median), with the kernel family that ran."""
+    import torch
+    from dataclasses import replace
+    from paper_2609_39185_b200 import ssdq
+    out = {"note": f"per-layer shape of config {cfg.index}, {layers} layers resident, {rounds} interleaved rounds of {reps} steps, median"}
+    ring = tuple(t[:, :layers].contiguous() for t in (xs, dts, Bs, Cs))
+    sin = ssdq.make_step_inputs(*ring, torch.empty_like(ring[0]))
+    for name in ("bf16", "fp16", "e4m3", "int8"):
+        fmt = {v: k for k, v in workloads.FORMAT_NAMES.items()}[name]
+        c = replace(cfg, n_layers=layers, fmt=fmt, scale_block=cfg.weyl_block if fmt in workloads.SCALED_FORMATS else 0)
+        stack = Stack(c, RULE_IDS["rtn"])
+        stack.run(1, 5, sin)
+        torch.cuda.synchronize()
+        times = {"rtn": [], "weyl": []}
+        for _ in range(rounds):
+            for rule in times:
+                stack.set_rule(RULE_IDS[rule])
+                times[rule].append(time_steps(stack, sin, 1, reps) / reps)
+        by = c.algorithmic_bytes_per_layer_step() * layers
+        med = {k: float(np.median(v)) for k, v in times.items()}
+        out[name] = {"rtn_gbs": by / med["rtn"] / 1e9, "weyl_gbs": by / med["weyl"] / 1e9, "rtn_frac": by / med["rtn"] / 1e9 / peak,
+                     "weyl_frac": by / med["weyl"] / 1e9 / peak, "weyl_over_rtn_time": med["weyl"] / med["rtn"],
+                     "bytes_per_entry": by / (layers * c.entries_per_layer), "kernel": ssdq.last_kernel()}
+        del stack
+        torch.cuda.empty_cache()
+    return out
 
 
 def sweep_batch(args, cfg):
@@ -326,7 +382,7 @@ def main():
             "pct_of_measured_copy": 100.0 * gbs / world / peak,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": None if (args.batch or args.format) else NCU_TRAFFIC_BYTES.get((cfg.index, args.rule)),
-                         "kernel": "ssd_update_tile_kernel" if cfg.headdim >= 32 and not cfg.a_per_state else "ssd_update_kernel", "peak_source": peak_src,
+                         "traffic_source": NCU_TRAFFIC_SOURCE, "kernel": ssdq.last_kernel(), "peak_source": peak_src,
                          "algorithmic_bytes_per_launch": bytes_per_launch, "launch_us": launch_secs * 1e6},
             "clocks": clocks, "gpu_launches": int(launches)}
 
@@ -340,7 +396,7 @@ def main():
             e0.record()
             for _ in range(reps):
                 for st in stack.states:
-                    dst.copy_(st)
+                    ssdq.copy(st, dst)
             e1.record()
             e1.synchronize()
             times["copy"].append(e0.elapsed_time(e1) / 1e3 / reps)
@@ -356,10 +412,14 @@ def main():
         line["sr_over_rtn_time"] = med["sr"] / med["rtn"]
         line["sr_hash_over_rtn_time"] = med["sr_hash"] / med["rtn"]
 
+        # ---- the other store formats on the same per-layer shape (2 layers resident: beyond L2), RTN against Weyl ----
+        if world == 1 and cfg.index == 5 and not (args.batch or args.format):
+            line["formats"] = formats_table(cfg, peak, xs, dts, Bs, Cs)
+
         # ---- end to end: per step, inputs come from pinned host memory and y goes back to the host ----
         in_bytes = sum(t[0].numel() * 4 for t in (xs_h, dts_h, Bs_h, Cs_h))
         out_bytes = ys[0].numel() * 4
-        e2e_steps = max(3, min(args.steps, 200))
+        e2e_steps = min(max(args.steps, 100), 400)      # at least 100 steps: a short run would time the pipeline's fill
         ys_ring_h = torch.empty(ys.shape, dtype=torch.float32, pin_memory=True)
         host_io = ssdq.make_step_inputs(xs_h, dts_h, Bs_h, Cs_h, ys_ring_h)
         slots = min(args.ring, 4)

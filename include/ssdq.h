@@ -1,12 +1,13 @@
 /* ssdq.h -- C ABI of the quantized selective-state-update decode library (CUDA, sm_100a).
  *
- * The library keeps a Mamba-style recurrent state in a low-precision store (FP16, BF16 or
- * FP8-E4M3 with an FP32 block scale) and, once per generated token and layer, makes one fused
- * pass over it: dequantise, h' = exp(dt*A)*h + dt*B*x (Eq. 1; Appendix B "Runners"), read out
- * y = C.h' + D*x from the unrounded h', and write h' back rounded by Eq. 2 under one of three
+ * The library keeps a Mamba-style recurrent state in a low-precision store -- FP16, BF16, FP8-E4M3
+ * with an FP32 block scale, or symmetric block-absmax integers INT8/7/6/4 with an FP32 block scale
+ * (Appendix B "Formats"); FP32 is the unrounded twin -- and, once per generated token and layer,
+ * makes one fused pass over it: dequantise, h' = exp(dt*A)*h + dt*B*x (Eq. 1; Appendix B "Runners"),
+ * read out y = C.h' + D*x from the unrounded h', and write h' back rounded by Eq. 2 under one of four
  * threshold rules (Section 2 "Rounding with a threshold"): round-to-nearest, stochastic rounding
- * driven by counter-based Philox4x32-10, or the golden-ratio Weyl dither in its 32-bit integer form
- * (Appendix B "Dithers").
+ * driven by counter-based Philox4x32-10 or by a cheap integer hash (Section 6.5 "Cost"), or the
+ * golden-ratio Weyl dither in its 32-bit integer form (Appendix B "Dithers").
  *
  * Conventions for every entry point
  *   - Pointers named in a descriptor are DEVICE pointers unless stated; descriptors themselves are
@@ -71,13 +72,13 @@ typedef struct {
 
 /* Fill `out` (HOST) for layer `layer` and offset seed `seed` (the paper's sigma; 0 in its runs).
  * `block` must be a positive multiple of 16.  Pure host arithmetic; no CUDA call. */
-int weyl_offsets_init(ssdq_weyl* out, uint32_t layer, uint32_t seed, uint32_t block);
+ssdq_status weyl_offsets_init(ssdq_weyl* out, uint32_t layer, uint32_t seed, uint32_t block);
 
 /* Test aid: write the 24-bit thresholds U of entries flat = first_flat .. first_flat + n - 1 at
  * write index step_t into out_u24 (DEVICE, n x uint32).  rule = SSDQ_WEYL uses `weyl`;
  * SSDQ_SR_PHILOX uses Philox4x32-10 with key = sr_seed and counter = (flat/4 low, flat/4 high,
  * step_t, layer), word flat % 4, top 24 bits; SSDQ_SR_HASH as defined at ssdq_rule; SSDQ_RTN writes zeros. */
-int ssdq_thresholds_materialize(int rule, const ssdq_weyl* weyl, uint64_t sr_seed, uint32_t layer,
+ssdq_status ssdq_thresholds_materialize(int rule, const ssdq_weyl* weyl, uint64_t sr_seed, uint32_t layer,
                                 uint64_t first_flat, uint64_t n, uint32_t step_t, uint32_t* out_u24, void* stream);
 
 /* One layer's decode-step problem. */
@@ -119,7 +120,7 @@ typedef struct {
  * exp_spec is the library's fixed binary32 exponential (clamp to [-87, 88], Cody-Waite reduction,
  * degree-7 polynomial), identical bit for bit on every call.  Values beyond the format's largest
  * finite number saturate to it; a value rounded to zero keeps its sign. */
-int ssd_state_update(const ssdq_update_desc* d, uint32_t step_t, void* stream);
+ssdq_status ssd_state_update(const ssdq_update_desc* d, uint32_t step_t, void* stream);
 
 /* Quantise an FP32 array into a store with the same rounding functions (Eq. 2): used to seed h_0
  * from a full-precision state (the paper quantises the end-of-prefill state) and to exercise the
@@ -127,7 +128,7 @@ int ssd_state_update(const ssdq_update_desc* d, uint32_t step_t, void* stream);
  * [n_rows, row_len] codes (16-byte aligned); dst_scales [n_rows, row_len / scale_block] for E4M3
  * else NULL.  row_len obeys the same limits as dstate; entry (row, col) has flat index
  * (row_index_base + row) * row_len + col. */
-int quantize_store(const float* src, void* dst_codes, float* dst_scales, uint64_t n_rows, uint32_t row_len,
+ssdq_status quantize_store(const float* src, void* dst_codes, float* dst_scales, uint64_t n_rows, uint32_t row_len,
                    uint32_t scale_block, int format, int rule, const ssdq_weyl* weyl, uint64_t sr_seed,
                    uint32_t layer, uint64_t row_index_base, uint32_t step_t, void* stream);
 
@@ -137,12 +138,12 @@ int quantize_store(const float* src, void* dst_codes, float* dst_scales, uint64_
  * its indices and step_t are those of quantize_store.  h' = fma(a, dequant(code), w) in binary32, then block scale,
  * threshold and Eq. 2 exactly as in ssd_state_update (whose state it reproduces bit for bit when fed a = exp_spec(dt*A)
  * and w = (dt*x)*B). */
-int ssd_replay_step(const float* w, const float* decay, uint32_t rows_per_decay, void* codes, float* scales, uint64_t n_rows,
+ssdq_status ssd_replay_step(const float* w, const float* decay, uint32_t rows_per_decay, void* codes, float* scales, uint64_t n_rows,
                     uint32_t row_len, uint32_t scale_block, int format, int rule, const ssdq_weyl* weyl, uint64_t sr_seed,
                     uint32_t layer, uint64_t row_index_base, uint32_t step_t, void* stream);
 
 /* Inverse view of a store: out[i] = decode(code[i]) (* scale[i / scale_block] for E4M3), DEVICE. */
-int ssdq_dequantize(const void* codes, const float* scales, uint64_t n, int format, uint32_t scale_block,
+ssdq_status ssdq_dequantize(const void* codes, const float* scales, uint64_t n, int format, uint32_t scale_block,
                     float* out, void* stream);
 
 /* Per-step inputs of the multi-step driver: element (t, l) of tensor X starts at
@@ -162,7 +163,7 @@ typedef struct {
  * t_first + n_steps - 1 and l = 0 .. n_layers - 1, one ssd_state_update launch of layers[l] with
  * write index t and the inputs of slot (t, l), all on `stream`, no host synchronisation.  The
  * x / dt / Bm / Cm / y / z members of layers[l] are ignored (taken from `in`). */
-int ssd_decode_run(const ssdq_update_desc* layers, uint32_t n_layers, uint32_t t_first, uint32_t n_steps,
+ssdq_status ssd_decode_run(const ssdq_update_desc* layers, uint32_t n_layers, uint32_t t_first, uint32_t n_steps,
                    const ssdq_step_inputs* in, void* stream);
 
 /* Replayable CUDA graph of the decode loop, for decode at small batch where the per-layer launches are bound by launch
@@ -175,10 +176,10 @@ int ssd_decode_run(const ssdq_update_desc* layers, uint32_t n_layers, uint32_t t
  * The results equal those of ssd_decode_run for the same write indices.  Creation allocates driver-side graph objects
  * (no device memory of the library's own). */
 typedef struct ssdq_graph ssdq_graph;
-int ssd_decode_graph_create(ssdq_graph** out, const ssdq_update_desc* layers, uint32_t n_layers, uint32_t steps_per_launch,
+ssdq_status ssd_decode_graph_create(ssdq_graph** out, const ssdq_update_desc* layers, uint32_t n_layers, uint32_t steps_per_launch,
                             const ssdq_step_inputs* in, uint32_t* step_counter);
-int ssd_decode_graph_launch(ssdq_graph* graph, void* stream);
-int ssd_decode_graph_destroy(ssdq_graph* graph);
+ssdq_status ssd_decode_graph_launch(ssdq_graph* graph, void* stream);
+ssdq_status ssd_decode_graph_destroy(ssdq_graph* graph);
 
 /* Periodic checkpointing (Section 6.5 "Periodic checkpointing"; Appendix B "Decode regime", CC = 8): the state lives in
  * full precision between checkpoints and only every `every`-th write, counted from t_first, is rounded into the store.
@@ -186,7 +187,7 @@ int ssd_decode_graph_destroy(ssdq_graph* graph);
  * dequantised store, or zeros for h_0 = 0).  Per step and layer: one FP32 update launch; on checkpoint steps also
  * quantize_store (work -> layers[l].state under the layer's rule at write index t) and ssdq_dequantize (store -> work).
  * With every == 1 the stores and y equal those of ssd_decode_run.  dstate <= 128. */
-int ssd_decode_run_checkpointed(const ssdq_update_desc* layers, float* const* work_fp32, uint32_t n_layers, uint32_t every,
+ssdq_status ssd_decode_run_checkpointed(const ssdq_update_desc* layers, float* const* work_fp32, uint32_t n_layers, uint32_t every,
                                 uint32_t t_first, uint32_t n_steps, const ssdq_step_inputs* in, void* stream);
 
 /* The same driver for callers whose per-step inputs and outputs live in HOST memory (the usual case when the
@@ -198,7 +199,7 @@ int ssd_decode_run_checkpointed(const ssdq_update_desc* layers, float* const* wo
  * t+1, compute of step t and copy-out of step t-1 overlap.  When all work enqueued on `stream` has completed,
  * every y has reached the host.  The state never leaves the device.  The two streams and the events are created
  * on the first call on a device (host-side driver resources, no device memory).  One call at a time per device. */
-int ssd_decode_run_host(const ssdq_update_desc* layers, uint32_t n_layers, uint32_t t_first, uint32_t n_steps,
+ssdq_status ssd_decode_run_host(const ssdq_update_desc* layers, uint32_t n_layers, uint32_t t_first, uint32_t n_steps,
                         const ssdq_step_inputs* host, const ssdq_step_inputs* staging, void* stream);
 
 /* Sanity metric of a quantised trajectory against its full-precision twin (Appendix B "Open-loop replay":
@@ -209,7 +210,7 @@ int ssd_decode_run_host(const ssdq_update_desc* layers, uint32_t n_layers, uint3
  * bytes, 16-byte aligned, owned by the caller; it holds per-(b, h) partial sums between the two passes (the sums
  * over the batch are taken in a fixed order, so results are identical from run to run). */
 uint64_t ssdq_state_error_workspace_bytes(uint32_t batch, uint32_t nheads);
-int ssdq_state_error(const void* codes, const float* scales, const float* twin, uint32_t batch, uint32_t nheads,
+ssdq_status ssdq_state_error(const void* codes, const float* scales, const float* twin, uint32_t batch, uint32_t nheads,
                      uint32_t headdim, uint32_t dstate, int format, uint32_t scale_block, double* err2_per_head,
                      double* ref2_per_head, void* workspace, uint64_t workspace_bytes, void* stream);
 
@@ -223,21 +224,33 @@ int ssdq_state_error(const void* codes, const float* scales, const float* twin, 
  * loads the library holds until the process exits.
  *   - batch * nheads beyond SSDQ_STATE_ERROR_STATIC_MAX_ITEMS is rejected with SSDQ_ERR_SHAPE (use ssdq_state_error).
  *   - The first call on each device looks up the array's address on that device (the device must be current);
- *     make that first call before any stream capture begins.
+ *     make that first call before any stream capture begins.  The address is kept for the life of the process:
+ *     it does not survive a cudaDeviceReset of that device.
  *   - All calls share the one array, which keeps the contents of the last call.  Nothing in it has to start at zero
  *     (each call overwrites every slot it later reads), but two calls that overlap on the GPU -- different streams,
  *     or different host threads on the same device -- race on it: serialise them.
  * Arguments and results are those of ssdq_state_error, minus the workspace. */
 #define SSDQ_STATE_ERROR_STATIC_MAX_ITEMS 65536u
-int ssdq_state_error_static(const void* codes, const float* scales, const float* twin, uint32_t batch, uint32_t nheads,
+ssdq_status ssdq_state_error_static(const void* codes, const float* scales, const float* twin, uint32_t batch, uint32_t nheads,
                             uint32_t headdim, uint32_t dstate, int format, uint32_t scale_block, double* err2_per_head,
                             double* ref2_per_head, void* stream);
 
 /* Surrogate of the paper's per-token KL (Section 4 "What we measure"; there is no vocabulary here): for each
  * sequence b, KL(p || q) = sum_i p_i log(p_i / q_i) with p = softmax(y_ref[b, :]) and q = softmax(y_q[b, :]) over the
  * `width` readout values of that sequence.  y_ref, y_q [batch, width] and kl_per_sequence [batch] are DEVICE floats. */
-int ssdq_readout_kl(const float* y_ref, const float* y_q, uint32_t batch, uint32_t width, float* kl_per_sequence,
+ssdq_status ssdq_readout_kl(const float* y_ref, const float* y_q, uint32_t batch, uint32_t width, float* kl_per_sequence,
                     void* stream);
+
+/* The floor of the timing protocol: a plain 128-bit copy of `bytes` bytes (a multiple of 16; both pointers DEVICE,
+ * 16-byte aligned, not overlapping) by a kernel of this library, so that a state update can be timed against a copy
+ * of the same buffers launched the same way (the "copy" column of Table 11, Section 6.5 "Cost"). */
+ssdq_status ssdq_copy(const void* src, void* dst, uint64_t bytes, void* stream);
+
+/* Name of the kernel family that the last fused-update launch issued from this thread used:
+ * "ssd_update_stream_kernel" (persistent, one-byte block-scaled stores on head-shaped tiles),
+ * "ssd_update_tile_kernel" (one CTA per head) or "ssd_update_kernel" (any shape); "" before the first launch.
+ * For benchmark records. */
+const char* ssdq_last_kernel(void);
 
 /* Text of the last error on this thread ("" if none).  The pointer stays valid until the next call
  * of the library on the same thread. */

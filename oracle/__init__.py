@@ -66,6 +66,8 @@ def lib() -> ctypes.CDLL:
         L.oracle_threshold.argtypes = [i32, u32, u32, u32, u64, u64, u32]
         L.oracle_round_array.restype = None
         L.oracle_round_array.argtypes = [vp, vp, u64, i32, i32, vp]
+        L.oracle_round_encode_array.restype = None
+        L.oracle_round_encode_array.argtypes = [vp, vp, u64, u64, i32, i32, vp]
         L.oracle_exp_spec_array.restype = None
         L.oracle_exp_spec_array.argtypes = [vp, u64, vp]
         L.oracle_state_update.restype = i32
@@ -139,6 +141,21 @@ def round_values(v, U, fmt, rule):
     out = np.empty_like(v)
     lib().oracle_round_array(_ptr(v), _ptr(U), v.size, fmt, rule, _ptr(out))
     return out
+
+
+def round_encode(v, U, fmt, rule):
+    """Codes of Eq. 2 applied to every entry of float32 `v` with thresholds `U` (an array like v, one integer for
+    all entries, or None under RTN): encode(round_values(v, U)) in one parallel pass."""
+    v = _f32(v)
+    codes = np.empty(v.shape, dtype=CODE_DTYPE[fmt])
+    if U is None:
+        Ua, nU = None, 0
+    else:
+        Ua = np.ascontiguousarray(np.atleast_1d(U), dtype=np.uint32)
+        nU = Ua.size
+        assert nU in (1, v.size)
+    lib().oracle_round_encode_array(_ptr(v), _ptr(Ua), nU, v.size, fmt, rule, _ptr(codes))
+    return codes
 
 
 def encode(q, fmt):

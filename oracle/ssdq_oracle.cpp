@@ -334,7 +334,17 @@ uint32_t oracle_threshold(int rule, uint32_t layer, uint32_t weyl_seed, uint32_t
     return threshold_u24(rp, flat, t);
 }
 void oracle_round_array(const float* v, const uint32_t* U, uint64_t n, int fmt, int rule, float* out) {
-    for (uint64_t i = 0; i < n; ++i) out[i] = round_on_grid(v[i], fmt, rule, U[i]);
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < (int64_t)n; ++i) out[i] = round_on_grid(v[i], fmt, rule, U[i]);
+}
+// Eq. 2 and the encoding, entry by entry, with the thresholds given: codes[i] = encode(round(v[i]; U[i])).
+// U may be null (RTN), or hold one value used for every entry (n_U == 1).
+void oracle_round_encode_array(const float* v, const uint32_t* U, uint64_t n_U, uint64_t n, int fmt, int rule, void* codes) {
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < (int64_t)n; ++i) {
+        const uint32_t u = U ? U[n_U == 1 ? 0 : i] : 0u;
+        store_code(codes, (uint64_t)i, fmt, encode(round_on_grid(v[i], fmt, rule, u), fmt));
+    }
 }
 void oracle_exp_spec_array(const float* z, uint64_t n, float* out) {
     for (uint64_t i = 0; i < n; ++i) out[i] = exp_spec(z[i]);

@@ -15,7 +15,7 @@ namespace {
 thread_local char g_err[256] = "";
 std::atomic<uint64_t> g_launches{0};
 
-int fail(int code, const char* fmt, ...) {
+ssdq_status fail(ssdq_status code, const char* fmt, ...) {
     va_list ap;
     va_start(ap, fmt);
     vsnprintf(g_err, sizeof(g_err), fmt, ap);
@@ -23,7 +23,7 @@ int fail(int code, const char* fmt, ...) {
     return code;
 }
 
-int cuda_result(cudaError_t e, const char* what) {
+ssdq_status cuda_result(cudaError_t e, const char* what) {
     if (e == cudaSuccess) { g_launches.fetch_add(1, std::memory_order_relaxed); return SSDQ_OK; }
     return fail(SSDQ_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
 }
@@ -57,7 +57,7 @@ ssdq::WeylConst weyl_const(const ssdq_weyl& w) {
 }
 
 // Checks shared by ssd_state_update and ssd_decode_run; per-step pointers are checked separately.
-int check_layer(const ssdq_update_desc* d) {
+ssdq_status check_layer(const ssdq_update_desc* d) {
     if (!d) return fail(SSDQ_ERR_NULL, "descriptor is NULL");
     if (d->batch == 0 || d->nheads == 0 || d->headdim == 0) return fail(SSDQ_ERR_SHAPE, "batch, nheads and headdim must be positive");
     if (!format_known(d->format)) return fail(SSDQ_ERR_UNSUPPORTED, "unknown format %d", d->format);
@@ -84,7 +84,7 @@ int check_layer(const ssdq_update_desc* d) {
     return SSDQ_OK;
 }
 
-int check_step_ptrs(const float* x, const float* dt, const float* Bm, const float* Cm, const float* y, const float* z = nullptr) {
+ssdq_status check_step_ptrs(const float* x, const float* dt, const float* Bm, const float* Cm, const float* y, const float* z = nullptr) {
     if (!x || !dt || !Bm || !Cm || !y) return fail(SSDQ_ERR_NULL, "x, dt, Bm, Cm and y are required");
     if (!aligned4(x) || !aligned4(dt) || !aligned4(y) || !aligned4(z)) return fail(SSDQ_ERR_ALIGN, "x, dt, y or z is misaligned");
     if (!aligned16(Bm) || !aligned16(Cm)) return fail(SSDQ_ERR_ALIGN, "Bm and Cm must be 16-byte aligned");
@@ -137,7 +137,7 @@ struct HostPipe {
 HostPipe g_pipes[64];
 std::mutex g_pipes_mutex;
 
-int host_pipe_for_current_device(HostPipe** out) {
+ssdq_status host_pipe_for_current_device(HostPipe** out) {
     int dev = -1;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return fail(SSDQ_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
@@ -162,14 +162,18 @@ int host_pipe_for_current_device(HostPipe** out) {
 
 }  // namespace
 
+namespace {
+thread_local int g_last_kernel = -1;
+}
 namespace ssdq {
-int report_failure(int status, const char* text) { return fail(status, "%s", text); }
+void note_kernel(int family) { g_last_kernel = family; }
+int report_failure(int status, const char* text) { return fail(static_cast<ssdq_status>(status), "%s", text); }
 void count_launches(unsigned n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 }  // namespace ssdq
 
 extern "C" {
 
-int weyl_offsets_init(ssdq_weyl* out, uint32_t layer, uint32_t seed, uint32_t block) {
+ssdq_status weyl_offsets_init(ssdq_weyl* out, uint32_t layer, uint32_t seed, uint32_t block) {
     if (!out) return fail(SSDQ_ERR_NULL, "out is NULL");
     if (block == 0 || block % 16 != 0) return fail(SSDQ_ERR_SHAPE, "block must be a positive multiple of 16");
     // Appendix B "Dithers": the decimal generators times 2^32, rounded to the nearest integer.
@@ -186,7 +190,7 @@ int weyl_offsets_init(ssdq_weyl* out, uint32_t layer, uint32_t seed, uint32_t bl
     return SSDQ_OK;
 }
 
-int ssdq_thresholds_materialize(int rule, const ssdq_weyl* weyl, uint64_t sr_seed, uint32_t layer, uint64_t first_flat,
+ssdq_status ssdq_thresholds_materialize(int rule, const ssdq_weyl* weyl, uint64_t sr_seed, uint32_t layer, uint64_t first_flat,
                                 uint64_t n, uint32_t step_t, uint32_t* out_u24, void* stream) {
     if (rule < SSDQ_RTN || rule > SSDQ_SR_HASH) return fail(SSDQ_ERR_UNSUPPORTED, "unknown rule %d", rule);
     if (n && !out_u24) return fail(SSDQ_ERR_NULL, "out_u24 is NULL");
@@ -201,8 +205,8 @@ int ssdq_thresholds_materialize(int rule, const ssdq_weyl* weyl, uint64_t sr_see
                                                static_cast<cudaStream_t>(stream)), "thresholds kernel");
 }
 
-int ssd_state_update(const ssdq_update_desc* d, uint32_t step_t, void* stream) {
-    int rc = check_layer(d);
+ssdq_status ssd_state_update(const ssdq_update_desc* d, uint32_t step_t, void* stream) {
+    ssdq_status rc = check_layer(d);
     if (rc != SSDQ_OK) return rc;
     rc = check_step_ptrs(d->x, d->dt, d->Bm, d->Cm, d->y, d->z);
     if (rc != SSDQ_OK) return rc;
@@ -211,7 +215,7 @@ int ssd_state_update(const ssdq_update_desc* d, uint32_t step_t, void* stream) {
                        "state-update kernel");
 }
 
-int quantize_store(const float* src, void* dst_codes, float* dst_scales, uint64_t n_rows, uint32_t row_len,
+ssdq_status quantize_store(const float* src, void* dst_codes, float* dst_scales, uint64_t n_rows, uint32_t row_len,
                    uint32_t scale_block, int format, int rule, const ssdq_weyl* weyl, uint64_t sr_seed, uint32_t layer,
                    uint64_t row_index_base, uint32_t step_t, void* stream) {
     if (!format_known(format)) return fail(SSDQ_ERR_UNSUPPORTED, "unknown format %d", format);
@@ -235,7 +239,7 @@ int quantize_store(const float* src, void* dst_codes, float* dst_scales, uint64_
     return cuda_result(ssdq::launch_quantize(p, kernel_format(format), rule, static_cast<cudaStream_t>(stream)), "quantize kernel");
 }
 
-int ssd_replay_step(const float* w, const float* decay, uint32_t rows_per_decay, void* codes, float* scales, uint64_t n_rows,
+ssdq_status ssd_replay_step(const float* w, const float* decay, uint32_t rows_per_decay, void* codes, float* scales, uint64_t n_rows,
                     uint32_t row_len, uint32_t scale_block, int format, int rule, const ssdq_weyl* weyl, uint64_t sr_seed,
                     uint32_t layer, uint64_t row_index_base, uint32_t step_t, void* stream) {
     if (!format_known(format)) return fail(SSDQ_ERR_UNSUPPORTED, "unknown format %d", format);
@@ -262,12 +266,12 @@ int ssd_replay_step(const float* w, const float* decay, uint32_t rows_per_decay,
                                              static_cast<cudaStream_t>(stream)), "replay kernel");
 }
 
-int ssd_decode_run_checkpointed(const ssdq_update_desc* layers, float* const* work_fp32, uint32_t n_layers, uint32_t every,
+ssdq_status ssd_decode_run_checkpointed(const ssdq_update_desc* layers, float* const* work_fp32, uint32_t n_layers, uint32_t every,
                                 uint32_t t_first, uint32_t n_steps, const ssdq_step_inputs* in, void* stream) {
     if (!layers || !in || !work_fp32) return fail(SSDQ_ERR_NULL, "layers, work_fp32 and in are required");
     if (n_layers == 0 || in->ring == 0 || every == 0) return fail(SSDQ_ERR_SHAPE, "n_layers, ring and every must be positive");
     for (uint32_t l = 0; l < n_layers; ++l) {
-        const int rc = check_layer(&layers[l]);
+        const ssdq_status rc = check_layer(&layers[l]);
         if (rc != SSDQ_OK) return rc;
         if (layers[l].format == SSDQ_FP32) return fail(SSDQ_ERR_UNSUPPORTED, "the store of a checkpointed run must be a quantised format");
         if (!work_fp32[l] || !aligned16(work_fp32[l])) return fail(SSDQ_ERR_ALIGN, "work_fp32[l] must be a 16-byte aligned device buffer");
@@ -277,7 +281,7 @@ int ssd_decode_run_checkpointed(const ssdq_update_desc* layers, float* const* wo
     for (uint32_t sl = 0; sl < slots; ++sl)
         for (uint32_t l = 0; l < n_layers; ++l) {
             const uint64_t k = (uint64_t)sl * n_layers + l;
-            const int rc = check_step_ptrs(in->x + k * in->stride_x, in->dt + k * in->stride_dt, in->Bm + k * in->stride_B,
+            const ssdq_status rc = check_step_ptrs(in->x + k * in->stride_x, in->dt + k * in->stride_dt, in->Bm + k * in->stride_B,
                                            in->Cm + k * in->stride_C, in->y + k * in->stride_y, in->z ? in->z + k * in->stride_z : nullptr);
             if (rc != SSDQ_OK) return rc;
         }
@@ -296,7 +300,7 @@ int ssd_decode_run_checkpointed(const ssdq_update_desc* layers, float* const* wo
             p.Cm = in->Cm + k * in->stride_C;
             p.y = in->y + k * in->stride_y;
             p.z = in->z ? in->z + k * in->stride_z : nullptr;
-            int rc = cuda_result(launch_update(p, SSDQ_FP32, SSDQ_RTN, d.a_per_state != 0, s), "state-update kernel");
+            ssdq_status rc = cuda_result(launch_update(p, SSDQ_FP32, SSDQ_RTN, d.a_per_state != 0, s), "state-update kernel");
             if (rc != SSDQ_OK) return rc;
             if ((i + 1) % every != 0) continue;
             // every `every`-th write is rounded into the store (Eq. 2 under the layer's rule) and read back
@@ -311,7 +315,7 @@ int ssd_decode_run_checkpointed(const ssdq_update_desc* layers, float* const* wo
     return SSDQ_OK;
 }
 
-int ssdq_dequantize(const void* codes, const float* scales, uint64_t n, int format, uint32_t scale_block, float* out,
+ssdq_status ssdq_dequantize(const void* codes, const float* scales, uint64_t n, int format, uint32_t scale_block, float* out,
                     void* stream) {
     if (!format_known(format)) return fail(SSDQ_ERR_UNSUPPORTED, "unknown format %d", format);
     if (n == 0) return SSDQ_OK;
@@ -324,12 +328,12 @@ int ssdq_dequantize(const void* codes, const float* scales, uint64_t n, int form
                        "dequantize kernel");
 }
 
-int ssd_decode_run(const ssdq_update_desc* layers, uint32_t n_layers, uint32_t t_first, uint32_t n_steps,
+ssdq_status ssd_decode_run(const ssdq_update_desc* layers, uint32_t n_layers, uint32_t t_first, uint32_t n_steps,
                    const ssdq_step_inputs* in, void* stream) {
     if (!layers || !in) return fail(SSDQ_ERR_NULL, "layers and in are required");
     if (n_layers == 0 || in->ring == 0) return fail(SSDQ_ERR_SHAPE, "n_layers and ring must be positive");
     for (uint32_t l = 0; l < n_layers; ++l) {
-        const int rc = check_layer(&layers[l]);
+        const ssdq_status rc = check_layer(&layers[l]);
         if (rc != SSDQ_OK) return rc;
     }
     // every slot of the ring is used with every layer: check the alignment of each (slot, layer) once
@@ -337,8 +341,8 @@ int ssd_decode_run(const ssdq_update_desc* layers, uint32_t n_layers, uint32_t t
     for (uint32_t s = 0; s < slots; ++s)
         for (uint32_t l = 0; l < n_layers; ++l) {
             const uint64_t k = (uint64_t)s * n_layers + l;
-            const int rc = check_step_ptrs(in->x + k * in->stride_x, in->dt + k * in->stride_dt, in->Bm + k * in->stride_B,
-                                           in->Cm + k * in->stride_C, in->y + k * in->stride_y);
+            const ssdq_status rc = check_step_ptrs(in->x + k * in->stride_x, in->dt + k * in->stride_dt, in->Bm + k * in->stride_B,
+                                                   in->Cm + k * in->stride_C, in->y + k * in->stride_y, in->z ? in->z + k * in->stride_z : nullptr);
             if (rc != SSDQ_OK) return rc;
         }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -353,7 +357,7 @@ int ssd_decode_run(const ssdq_update_desc* layers, uint32_t n_layers, uint32_t t
             p.Cm = in->Cm + k * in->stride_C;
             p.y = in->y + k * in->stride_y;
             p.z = in->z ? in->z + k * in->stride_z : nullptr;
-            const int rc = cuda_result(launch_update(p, layers[l].format, layers[l].rule, layers[l].a_per_state != 0, s),
+            const ssdq_status rc = cuda_result(launch_update(p, layers[l].format, layers[l].rule, layers[l].a_per_state != 0, s),
                                        "state-update kernel");
             if (rc != SSDQ_OK) return rc;
         }
@@ -363,7 +367,7 @@ int ssd_decode_run(const ssdq_update_desc* layers, uint32_t n_layers, uint32_t t
 
 uint64_t ssdq_state_error_workspace_bytes(uint32_t batch, uint32_t nheads) { return (uint64_t)batch * nheads * 16u; }
 
-int ssdq_state_error(const void* codes, const float* scales, const float* twin, uint32_t batch, uint32_t nheads,
+ssdq_status ssdq_state_error(const void* codes, const float* scales, const float* twin, uint32_t batch, uint32_t nheads,
                      uint32_t headdim, uint32_t dstate, int format, uint32_t scale_block, double* err2_per_head,
                      double* ref2_per_head, void* workspace, uint64_t workspace_bytes, void* stream) {
     if (!format_known(format)) return fail(SSDQ_ERR_UNSUPPORTED, "unknown format %d", format);
@@ -375,21 +379,21 @@ int ssdq_state_error(const void* codes, const float* scales, const float* twin, 
     if (workspace_bytes < ssdq_state_error_workspace_bytes(batch, nheads)) return fail(SSDQ_ERR_SHAPE, "workspace too small");
     if (format_scaled(format) && (!scales || scale_block == 0 || scale_block % 16 != 0))
         return fail(SSDQ_ERR_SHAPE, "scaled stores need scales and a scale_block that is a multiple of 16");
-    const int rc = cuda_result(ssdq::launch_state_error(codes, scales, twin, batch, nheads, headdim * dstate, kernel_format(format), scale_block,
+    const ssdq_status rc = cuda_result(ssdq::launch_state_error(codes, scales, twin, batch, nheads, headdim * dstate, kernel_format(format), scale_block,
                                                         err2_per_head, ref2_per_head, workspace, static_cast<cudaStream_t>(stream)),
                                "state-error kernels");
     if (rc == SSDQ_OK) g_launches.fetch_add(1, std::memory_order_relaxed);   // two kernels per call
     return rc;
 }
 
-int ssdq_readout_kl(const float* y_ref, const float* y_q, uint32_t batch, uint32_t width, float* kl_per_sequence, void* stream) {
+ssdq_status ssdq_readout_kl(const float* y_ref, const float* y_q, uint32_t batch, uint32_t width, float* kl_per_sequence, void* stream) {
     if (batch == 0 || width == 0) return fail(SSDQ_ERR_SHAPE, "batch and width must be positive");
     if (!y_ref || !y_q || !kl_per_sequence) return fail(SSDQ_ERR_NULL, "y_ref, y_q and kl_per_sequence are required");
     return cuda_result(ssdq::launch_readout_kl(y_ref, y_q, batch, width, kl_per_sequence, static_cast<cudaStream_t>(stream)),
                        "readout-KL kernel");
 }
 
-int ssd_decode_run_host(const ssdq_update_desc* layers, uint32_t n_layers, uint32_t t_first, uint32_t n_steps,
+ssdq_status ssd_decode_run_host(const ssdq_update_desc* layers, uint32_t n_layers, uint32_t t_first, uint32_t n_steps,
                         const ssdq_step_inputs* host, const ssdq_step_inputs* staging, void* stream) {
     if (!layers || !host || !staging) return fail(SSDQ_ERR_NULL, "layers, host and staging are required");
     if (n_layers == 0 || host->ring == 0) return fail(SSDQ_ERR_SHAPE, "n_layers and host ring must be positive");
@@ -399,22 +403,24 @@ int ssd_decode_run_host(const ssdq_update_desc* layers, uint32_t n_layers, uint3
         (host->z == nullptr) != (staging->z == nullptr))
         return fail(SSDQ_ERR_SHAPE, "host and staging strides must be equal");
     if (!host->x || !host->dt || !host->Bm || !host->Cm || !host->y) return fail(SSDQ_ERR_NULL, "host x, dt, Bm, Cm and y are required");
+    if (!aligned4(host->x) || !aligned4(host->dt) || !aligned4(host->Bm) || !aligned4(host->Cm) || !aligned4(host->y) || !aligned4(host->z))
+        return fail(SSDQ_ERR_ALIGN, "host arrays must be 4-byte aligned");
     for (uint32_t l = 0; l < n_layers; ++l) {
-        const int rc = check_layer(&layers[l]);
+        const ssdq_status rc = check_layer(&layers[l]);
         if (rc != SSDQ_OK) return rc;
     }
     for (uint32_t sl = 0; sl < staging->ring; ++sl)
         for (uint32_t l = 0; l < n_layers; ++l) {
             const uint64_t k = (uint64_t)sl * n_layers + l;
-            const int rc = check_step_ptrs(staging->x + k * staging->stride_x, staging->dt + k * staging->stride_dt,
+            const ssdq_status rc = check_step_ptrs(staging->x + k * staging->stride_x, staging->dt + k * staging->stride_dt,
                                            staging->Bm + k * staging->stride_B, staging->Cm + k * staging->stride_C,
-                                           staging->y + k * staging->stride_y);
+                                           staging->y + k * staging->stride_y, staging->z ? staging->z + k * staging->stride_z : nullptr);
             if (rc != SSDQ_OK) return rc;
         }
     if (n_steps == 0) return SSDQ_OK;
     cudaStream_t compute = static_cast<cudaStream_t>(stream);
     HostPipe* hp = nullptr;
-    int rc = host_pipe_for_current_device(&hp);
+    ssdq_status rc = host_pipe_for_current_device(&hp);
     if (rc != SSDQ_OK) return rc;
     std::lock_guard<std::mutex> lock(hp->mutex);
 #define SSDQ_TRY(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return fail(SSDQ_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_)); } while (0)
@@ -476,7 +482,7 @@ struct ssdq_graph {
     uint32_t steps = 0, n_layers = 0;
 };
 
-int ssd_decode_graph_create(ssdq_graph** out, const ssdq_update_desc* layers, uint32_t n_layers, uint32_t steps_per_launch,
+ssdq_status ssd_decode_graph_create(ssdq_graph** out, const ssdq_update_desc* layers, uint32_t n_layers, uint32_t steps_per_launch,
                             const ssdq_step_inputs* in, uint32_t* step_counter) {
     if (!out || !layers || !in || !step_counter) return fail(SSDQ_ERR_NULL, "out, layers, in and step_counter are required");
     *out = nullptr;
@@ -484,13 +490,13 @@ int ssd_decode_graph_create(ssdq_graph** out, const ssdq_update_desc* layers, ui
     if (steps_per_launch % in->ring != 0) return fail(SSDQ_ERR_SHAPE, "steps_per_launch must be a multiple of the input ring");
     if (!aligned4(step_counter)) return fail(SSDQ_ERR_ALIGN, "step_counter is misaligned");
     for (uint32_t l = 0; l < n_layers; ++l) {
-        const int rc = check_layer(&layers[l]);
+        const ssdq_status rc = check_layer(&layers[l]);
         if (rc != SSDQ_OK) return rc;
     }
     for (uint32_t sl = 0; sl < in->ring; ++sl)
         for (uint32_t l = 0; l < n_layers; ++l) {
             const uint64_t k = (uint64_t)sl * n_layers + l;
-            const int rc = check_step_ptrs(in->x + k * in->stride_x, in->dt + k * in->stride_dt, in->Bm + k * in->stride_B,
+            const ssdq_status rc = check_step_ptrs(in->x + k * in->stride_x, in->dt + k * in->stride_dt, in->Bm + k * in->stride_B,
                                            in->Cm + k * in->stride_C, in->y + k * in->stride_y, in->z ? in->z + k * in->stride_z : nullptr);
             if (rc != SSDQ_OK) return rc;
         }
@@ -500,7 +506,7 @@ int ssd_decode_graph_create(ssdq_graph** out, const ssdq_update_desc* layers, ui
     ssdq_graph* g = new ssdq_graph();
     g->steps = steps_per_launch;
     g->n_layers = n_layers;
-    int rc = SSDQ_OK;
+    ssdq_status rc = SSDQ_OK;
     e = cudaStreamBeginCapture(cs, cudaStreamCaptureModeThreadLocal);
     if (e != cudaSuccess) rc = fail(SSDQ_ERR_CUDA, "cudaStreamBeginCapture: %s", cudaGetErrorString(e));
     if (rc == SSDQ_OK) {
@@ -540,7 +546,7 @@ int ssd_decode_graph_create(ssdq_graph** out, const ssdq_update_desc* layers, ui
     return SSDQ_OK;
 }
 
-int ssd_decode_graph_launch(ssdq_graph* g, void* stream) {
+ssdq_status ssd_decode_graph_launch(ssdq_graph* g, void* stream) {
     if (!g || !g->exec) return fail(SSDQ_ERR_NULL, "graph handle is NULL");
     const cudaError_t e = cudaGraphLaunch(g->exec, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return fail(SSDQ_ERR_CUDA, "cudaGraphLaunch: %s", cudaGetErrorString(e));
@@ -548,12 +554,29 @@ int ssd_decode_graph_launch(ssdq_graph* g, void* stream) {
     return SSDQ_OK;
 }
 
-int ssd_decode_graph_destroy(ssdq_graph* g) {
+ssdq_status ssd_decode_graph_destroy(ssdq_graph* g) {
     if (!g) return SSDQ_OK;
     if (g->exec) cudaGraphExecDestroy(g->exec);
     if (g->graph) cudaGraphDestroy(g->graph);
     delete g;
     return SSDQ_OK;
+}
+
+ssdq_status ssdq_copy(const void* src, void* dst, uint64_t bytes, void* stream) {
+    if (bytes == 0) return SSDQ_OK;
+    if (!src || !dst) return fail(SSDQ_ERR_NULL, "src and dst are required");
+    if (bytes % 16 != 0) return fail(SSDQ_ERR_SHAPE, "bytes must be a multiple of 16");
+    if (!aligned16(src) || !aligned16(dst)) return fail(SSDQ_ERR_ALIGN, "src and dst must be 16-byte aligned");
+    return cuda_result(ssdq::launch_copy(src, dst, bytes, static_cast<cudaStream_t>(stream)), "copy kernel");
+}
+
+const char* ssdq_last_kernel(void) {
+    switch (g_last_kernel) {
+        case 0: return "ssd_update_kernel";
+        case 1: return "ssd_update_tile_kernel";
+        case 2: return "ssd_update_stream_kernel";
+        default: return "";
+    }
 }
 
 const char* ssdq_last_error(void) { return g_err; }

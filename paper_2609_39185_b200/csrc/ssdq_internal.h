@@ -74,8 +74,10 @@ cudaError_t launch_state_error(const void* codes, const float* scales, const flo
                                void* workspace, cudaStream_t s);
 // error text / launch counter of the C ABI, for entry points defined outside ssdq_api.cu
 int report_failure(int status, const char* text);
+void note_kernel(int family);      // 0 generic, 1 tile, 2 stream: which fused-update kernel the launcher picked
 void count_launches(unsigned n);
 
+cudaError_t launch_copy(const void* src, void* dst, uint64_t bytes, cudaStream_t s);
 cudaError_t launch_counter_add(uint32_t* counter, uint32_t n, cudaStream_t s);
 cudaError_t launch_readout_kl(const float* y_ref, const float* y_q, uint32_t batch, uint32_t width, float* kl, cudaStream_t s);
 

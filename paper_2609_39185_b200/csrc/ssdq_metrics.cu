@@ -124,6 +124,24 @@ __global__ void __launch_bounds__(kMetricThreads) readout_kl_kernel(const float*
     if (threadIdx.x == 0) kl[blockIdx.x] = (float)acc;
 }
 
+// Plain 128-bit copy, grid-stride, one wave of CTAs: the floor that a state update is timed against (Table 11, "copy").
+__global__ void __launch_bounds__(256) copy_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, uint64_t n_vec) {
+    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (; i + 3 * stride < n_vec; i += 4 * stride) {          // four independent loads in flight per thread
+        const uint4 a = src[i], b = src[i + stride], c = src[i + 2 * stride], d = src[i + 3 * stride];
+        dst[i] = a; dst[i + stride] = b; dst[i + 2 * stride] = c; dst[i + 3 * stride] = d;
+    }
+    for (; i < n_vec; i += stride) dst[i] = src[i];
+}
+cudaError_t launch_copy(const void* src, void* dst, uint64_t bytes, cudaStream_t s) {
+    const uint64_t n_vec = bytes / 16;
+    uint64_t grid = (n_vec + 255) / 256;
+    if (grid > 148u * 8u) grid = 148u * 8u;
+    copy_kernel<<<(unsigned)grid, 256, 0, s>>>(static_cast<const uint4*>(src), static_cast<uint4*>(dst), n_vec);
+    return cudaGetLastError();
+}
+
 __global__ void counter_add_kernel(uint32_t* counter, uint32_t n) { *counter += n; }
 cudaError_t launch_counter_add(uint32_t* counter, uint32_t n, cudaStream_t s) {
     counter_add_kernel<<<1, 1, 0, s>>>(counter, n);
@@ -153,16 +171,16 @@ double2* g_static_ptr[kMaxDevices] = {};     // device address of g_static_parti
 
 // In host code the name g_static_partials is only a stand-in for the symbol, not a device address: the
 // address valid on the current device has to be asked for.  Done once per device, on the first call there.
-int static_scratch_for_current_device(double2** out) {
+ssdq_status static_scratch_for_current_device(double2** out) {
     int dev = -1;
     cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return ssdq::report_failure(SSDQ_ERR_CUDA, cudaGetErrorString(e));
-    if (dev < 0 || dev >= kMaxDevices) return ssdq::report_failure(SSDQ_ERR_UNSUPPORTED, "device ordinal beyond the static table");
+    if (e != cudaSuccess) return (ssdq_status)ssdq::report_failure(SSDQ_ERR_CUDA, cudaGetErrorString(e));
+    if (dev < 0 || dev >= kMaxDevices) return (ssdq_status)ssdq::report_failure(SSDQ_ERR_UNSUPPORTED, "device ordinal beyond the static table");
     std::lock_guard<std::mutex> lock(g_static_mutex);
     if (!g_static_ptr[dev]) {
         void* ptr = nullptr;
         e = cudaGetSymbolAddress(&ptr, g_static_partials);
-        if (e != cudaSuccess || !ptr) return ssdq::report_failure(SSDQ_ERR_CUDA, e != cudaSuccess ? cudaGetErrorString(e) : "no address for the static scratch");
+        if (e != cudaSuccess || !ptr) return (ssdq_status)ssdq::report_failure(SSDQ_ERR_CUDA, e != cudaSuccess ? cudaGetErrorString(e) : "no address for the static scratch");
         g_static_ptr[dev] = static_cast<double2*>(ptr);
     }
     *out = g_static_ptr[dev];
@@ -171,29 +189,29 @@ int static_scratch_for_current_device(double2** out) {
 
 }  // namespace
 
-extern "C" int ssdq_state_error_static(const void* codes, const float* scales, const float* twin, uint32_t batch,
+extern "C" ssdq_status ssdq_state_error_static(const void* codes, const float* scales, const float* twin, uint32_t batch,
                                        uint32_t nheads, uint32_t headdim, uint32_t dstate, int format,
                                        uint32_t scale_block, double* err2_per_head, double* ref2_per_head, void* stream) {
-    if (format < SSDQ_FP16 || format > SSDQ_INT4) return ssdq::report_failure(SSDQ_ERR_UNSUPPORTED, "unknown format");
-    if (batch == 0 || nheads == 0 || headdim == 0 || dstate == 0) return ssdq::report_failure(SSDQ_ERR_SHAPE, "sizes must be positive");
-    if (((uint64_t)headdim * dstate) % 16 != 0) return ssdq::report_failure(SSDQ_ERR_SHAPE, "headdim * dstate must be a multiple of 16");
+    if (format < SSDQ_FP16 || format > SSDQ_INT4) return (ssdq_status)ssdq::report_failure(SSDQ_ERR_UNSUPPORTED, "unknown format");
+    if (batch == 0 || nheads == 0 || headdim == 0 || dstate == 0) return (ssdq_status)ssdq::report_failure(SSDQ_ERR_SHAPE, "sizes must be positive");
+    if (((uint64_t)headdim * dstate) % 16 != 0) return (ssdq_status)ssdq::report_failure(SSDQ_ERR_SHAPE, "headdim * dstate must be a multiple of 16");
     if ((uint64_t)batch * nheads > kStaticMaxItems)
-        return ssdq::report_failure(SSDQ_ERR_SHAPE, "batch * nheads exceeds SSDQ_STATE_ERROR_STATIC_MAX_ITEMS (65536): "
+        return (ssdq_status)ssdq::report_failure(SSDQ_ERR_SHAPE, "batch * nheads exceeds SSDQ_STATE_ERROR_STATIC_MAX_ITEMS (65536): "
                                                    "use ssdq_state_error with a caller-owned workspace");
-    if (!codes || !twin || !err2_per_head || !ref2_per_head) return ssdq::report_failure(SSDQ_ERR_NULL, "codes, twin and outputs are required");
+    if (!codes || !twin || !err2_per_head || !ref2_per_head) return (ssdq_status)ssdq::report_failure(SSDQ_ERR_NULL, "codes, twin and outputs are required");
     if ((reinterpret_cast<uintptr_t>(codes) & 15u) || (reinterpret_cast<uintptr_t>(twin) & 3u))
-        return ssdq::report_failure(SSDQ_ERR_ALIGN, "codes must be 16-byte aligned");
+        return (ssdq_status)ssdq::report_failure(SSDQ_ERR_ALIGN, "codes must be 16-byte aligned");
     const bool scaled = format == SSDQ_E4M3 || format >= SSDQ_INT8;
     if (scaled && (!scales || scale_block == 0 || scale_block % 16 != 0))
-        return ssdq::report_failure(SSDQ_ERR_SHAPE, "scaled stores need scales and a scale_block that is a multiple of 16");
+        return (ssdq_status)ssdq::report_failure(SSDQ_ERR_SHAPE, "scaled stores need scales and a scale_block that is a multiple of 16");
     double2* scratch = nullptr;
-    const int rc = static_scratch_for_current_device(&scratch);
+    const ssdq_status rc = static_scratch_for_current_device(&scratch);
     if (rc != SSDQ_OK) return rc;
     // every partial the second pass reads is written by the first pass of this same call: nothing has to be cleared
     const cudaError_t e = ssdq::launch_state_error(codes, scales, twin, batch, nheads, headdim * dstate,
                                                    format >= SSDQ_INT8 ? (int)ssdq::FMT_INT : format, scale_block,
                                                    err2_per_head, ref2_per_head, scratch, static_cast<cudaStream_t>(stream));
-    if (e != cudaSuccess) return ssdq::report_failure(SSDQ_ERR_CUDA, cudaGetErrorString(e));
+    if (e != cudaSuccess) return (ssdq_status)ssdq::report_failure(SSDQ_ERR_CUDA, cudaGetErrorString(e));
     ssdq::count_launches(2);
     return SSDQ_OK;
 }

@@ -22,34 +22,6 @@
 
 namespace ssdq {
 
-// ---- two binary32 values in one 64-bit register pair ------------------------------------------------------------
-typedef unsigned long long f32x2;
-__device__ __forceinline__ f32x2 pack2(float lo, float hi) { f32x2 r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi)); return r; }
-__device__ __forceinline__ f32x2 pack2u(uint32_t lo, uint32_t hi) { f32x2 r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi)); return r; }
-__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
-__device__ __forceinline__ void unpack2u(f32x2 v, uint32_t& lo, uint32_t& hi) { asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v)); }
-__device__ __forceinline__ f32x2 mul2_rn(f32x2 a, f32x2 b) { f32x2 r; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
-__device__ __forceinline__ f32x2 add2_rn(f32x2 a, f32x2 b) { f32x2 r; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
-__device__ __forceinline__ f32x2 add2_rm(f32x2 a, f32x2 b) { f32x2 r; asm("add.rm.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
-__device__ __forceinline__ f32x2 fma2_rn(f32x2 a, f32x2 b, f32x2 c) { f32x2 r; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c)); return r; }
-__device__ __forceinline__ f32x2 fma2_rm(f32x2 a, f32x2 b, f32x2 c) { f32x2 r; asm("fma.rm.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c)); return r; }
-// max(m, |a|, |b|) and min(m, |a|, |b|) in one instruction
-__device__ __forceinline__ float max3abs(float m, float a, float b) { float r; asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(m), "f"(fabsf(a)), "f"(fabsf(b))); return r; }
-__device__ __forceinline__ float min3abs(float m, float a, float b) { float r; asm("min.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(m), "f"(fabsf(a)), "f"(fabsf(b))); return r; }
-
-// amax / top, correctly rounded, for the constant tops of the scaled stores (448, 127, 63, 31, 7): with c = RN(1/top),
-// q = RN(amax c), r = amax - top q (exact in one fma) and RN(q + r c) is the correctly rounded quotient -- checked
-// against IEEE division for every binary32 significand and each of the five constants.  A small amax is scaled by
-// 2^64 first so that no intermediate underflows; scaling back rounds only when the quotient is below the smallest
-// normal number, where the caller's floor at that number hides it.  Only for max(result, FLT_MIN).
-__device__ __forceinline__ float div_by_top(float amax, float top, float inv_top) {
-    const bool small = amax < 0x1p-60f;
-    const float a = __fmul_rn(amax, small ? 0x1p64f : 1.0f);
-    const float q = __fmul_rn(a, inv_top);
-    const float r = __fmaf_rn(__fmaf_rn(-top, q, a), inv_top, q);
-    return __fmul_rn(r, small ? 0x1p-64f : 1.0f);
-}
-
 // Unpack one 32-bit word of one-byte codes into two packed pairs (exact widening).
 __device__ __forceinline__ void unpack4_e4m3_x2(uint32_t w, f32x2& p01, f32x2& p23) {
     float f[4];
@@ -62,103 +34,6 @@ __device__ __forceinline__ void unpack4_int8_x2(uint32_t w, f32x2& p01, f32x2& p
     const f32x2 off = pack2(-8388736.0f, -8388736.0f);     // -(2^23 + 128)
     p01 = add2_rn(pack2u(__byte_perm(w, 0x4B000000u, 0x7540), __byte_perm(w, 0x4B000000u, 0x7541)), off);
     p23 = add2_rn(pack2u(__byte_perm(w, 0x4B000000u, 0x7542), __byte_perm(w, 0x4B000000u, 0x7543)), off);
-}
-
-// ---- rounding of a lane's 16 scaled values (8 packed pairs) into 16 one-byte codes ------------------------------
-// four binary32 values -> four E4M3 codes in memory order (v0 in the low byte), round to nearest even, saturating
-__device__ __forceinline__ uint32_t rtn_pack4_e4m3(float v0, float v1, float v2, float v3) {
-    uint32_t r;
-    asm("{.reg .b16 lo, hi; cvt.rn.satfinite.e4m3x2.f32 lo, %2, %1; cvt.rn.satfinite.e4m3x2.f32 hi, %4, %3; mov.b32 %0, {lo, hi};}"
-        : "=r"(r) : "f"(v0), "f"(v1), "f"(v2), "f"(v3));
-    return r;
-}
-// The stochastic-rounding convert with all random bits zero adds nothing and truncates the magnitude onto the E4M3
-// grid (subnormal targets and saturation included: compared with the exact convert of the truncated value on every
-// binary32 pattern).  Its first operand lands in the HIGH byte.
-__device__ __forceinline__ uint32_t trunc_pack4_e4m3(float v0, float v1, float v2, float v3) {
-    uint32_t r;
-    asm("cvt.rs.satfinite.e4m3x4.f32 %0, {%1, %2, %3, %4}, %5;" : "=r"(r) : "f"(v3), "f"(v2), "f"(v1), "f"(v0), "r"(0u));
-    return r;
-}
-
-// acc[k]: the threshold word of entry k (U = acc >> 8); unused under RTN.
-template <int FMT, int RULE>
-__device__ __forceinline__ uint4 round_pack_lane_x2(const f32x2* v2, const uint32_t* acc, float qmax, float vmin) {
-    uint32_t w[4];
-    if constexpr (RULE == RULE_RTN) {
-        if constexpr (FMT == FMT_E4M3) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                float a, b, c, d;
-                unpack2(v2[2 * i], a, b);
-                unpack2(v2[2 * i + 1], c, d);
-                w[i] = rtn_pack4_e4m3(a, b, c, d);
-            }
-        } else {
-            const f32x2 magic = pack2(kIntMagic, kIntMagic);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                uint32_t t0, t1, t2, t3;
-                unpack2u(add2_rn(v2[2 * i], magic), t0, t1);         // nearest-even integer in the low mantissa bits
-                unpack2u(add2_rn(v2[2 * i + 1], magic), t2, t3);
-                w[i] = pack4_low_bytes(t0, t1, t2, t3);
-            }
-        }
-    } else if constexpr (FMT == FMT_INT) {
-        // clamp(floor(v + u)): the sum rounded down, then the add of the magic floors it (Eq. 2 on the integer grid);
-        // the integers sit in the low halves of the sums, where they are clamped two at a time
-        const f32x2 magic = pack2(kIntMagic, kIntMagic), ulp = pack2(0x1p-32f, 0x1p-32f);
-        const uint32_t q = (uint32_t)(int)qmax, hi2 = q | (q << 16), lo2 = (uint32_t)(-(int)q & 0xFFFF) * 0x00010001u;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            uint32_t kk[2];
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int k = 4 * i + 2 * h;
-                const f32x2 u2 = pack2(__uint2float_rn(acc[k] & 0xFFFFFF00u), __uint2float_rn(acc[k + 1] & 0xFFFFFF00u));   // exact: 24 bits
-                uint32_t t0, t1;
-                unpack2u(add2_rm(fma2_rm(u2, ulp, v2[k / 2]), magic), t0, t1);
-                kk[h] = __vimax3_s16x2(__vimin3_s16x2(__byte_perm(t0, t1, 0x5410), hi2, hi2), lo2, lo2);
-            }
-            w[i] = __byte_perm(kk[0], kk[1], 0x6420);
-        }
-    } else {
-        // E4M3 dither.  Every |v| >= 2^-6 has an E4M3 target in the normal range: 20 binary32 mantissa bits are
-        // dropped, and floor(v / 2^q + u) adds the leading 20 bits of (threshold XOR sign mask) to the sign-magnitude
-        // bits and truncates; the carry crosses binades by itself and the convert saturates.  A lane with a smaller
-        // value (zero included) takes Eq. 2 literally in binary32 instead.
-        if (vmin >= 0x1p-6f) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                float r[4];
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t b0, b1;
-                    unpack2u(v2[2 * i + h], b0, b1);
-                    const int k = 4 * i + 2 * h;
-                    const uint32_t x0 = acc[k] ^ (uint32_t)((int32_t)b0 >> 31), x1 = acc[k + 1] ^ (uint32_t)((int32_t)b1 >> 31);
-                    r[2 * h] = __uint_as_float(b0 + (x0 >> 12));
-                    r[2 * h + 1] = __uint_as_float(b1 + (x1 >> 12));
-                }
-                w[i] = trunc_pack4_e4m3(r[0], r[1], r[2], r[3]);
-            }
-        } else {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                float r[4], vv[4];
-                unpack2(v2[2 * i], vv[0], vv[1]);
-                unpack2(v2[2 * i + 1], vv[2], vv[3]);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const float scale = dither_step_scale<3, -6, 127>(vv[j]);
-                    const float q = floor_to_step(dithered_sum_rm(vv[j], acc[4 * i + j], scale), scale);
-                    r[j] = __uint_as_float((__float_as_uint(q) & 0x7FFFFFFFu) | (__float_as_uint(vv[j]) & 0x80000000u));
-                }
-                w[i] = rtn_pack4_e4m3(r[0], r[1], r[2], r[3]);   // exact; saturates beyond 448
-            }
-        }
-    }
-    return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
 __device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gmem_src) {
@@ -332,19 +207,9 @@ __global__ void __launch_bounds__(kThreads, SSDQ_STREAM_MINB) ssd_update_stream_
             const float s = fmaxf(div_by_top(amax, top, inv_top), 1.17549435e-38f);
             const float rinv = __frcp_rn(s);
             const f32x2 rinv2 = pack2(rinv, rinv);
-            float vminA = 3.0e38f, vminB = 3.0e38f;
+            float v[EPL];
 #pragma unroll
-            for (int i = 0; i < EPL / 2; i += 2) {
-                hv[i] = mul2_rn(hv[i], rinv2);
-                hv[i + 1] = mul2_rn(hv[i + 1], rinv2);
-                if constexpr (FMT == FMT_E4M3 && RULE != RULE_RTN) {
-                    float e0, e1, e2, e3;
-                    unpack2(hv[i], e0, e1);
-                    unpack2(hv[i + 1], e2, e3);
-                    vminA = min3abs(vminA, e0, e1);
-                    vminB = min3abs(vminB, e2, e3);
-                }
-            }
+            for (int i = 0; i < EPL / 2; ++i) unpack2(mul2_rn(hv[i], rinv2), v[2 * i], v[2 * i + 1]);
             if constexpr (ROW_SCALE) { if (lis == 0) c_sc[k] = s; }
             else c_sc[k * SPR] = s;
 
@@ -365,7 +230,7 @@ __global__ void __launch_bounds__(kThreads, SSDQ_STREAM_MINB) ssd_update_stream_
                 }
                 grp_row += N / 4;
             }
-            c_codes[k * LPR] = round_pack_lane_x2<FMT, RULE>(hv, acc, top, fminf(vminA, vminB));
+            c_codes[k * LPR] = round_pack16<FMT, RULE>(v, acc, top);
             return __fadd_rn(d0, d1);
         };
 #pragma unroll
@@ -426,6 +291,7 @@ inline cudaError_t launch_stream(const UpdateParams& p, cudaStream_t stream) {
     if (e != cudaSuccess) return e;
     uint32_t grid = (uint32_t)(ctas * sms);            // one wave of resident CTAs
     if (grid > p.n_items) grid = p.n_items;
+    note_kernel(2);
     ssd_update_stream_kernel<FMT, RULE, LPR, RPS, STAGES, ROW_SCALE><<<grid, kThreads, stream_smem_bytes<RPS, STAGES>(), stream>>>(p);
     return cudaGetLastError();
 }

@@ -62,15 +62,8 @@ __device__ __forceinline__ uint4 round_pack_lane(const float* v, uint32_t acc0, 
         } else if constexpr (FMT == FMT_BF16) {
 #pragma unroll
             for (int i = 0; i < 4; ++i) w[i] = rtn_pack2_bf16(v[2 * i], v[2 * i + 1]);
-        } else if constexpr (FMT == FMT_INT) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-                w[i] = pack4_low_bytes(int_rtn_biased(v[4 * i], qmax), int_rtn_biased(v[4 * i + 1], qmax),
-                                       int_rtn_biased(v[4 * i + 2], qmax), int_rtn_biased(v[4 * i + 3], qmax));
         } else {
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-                w[i] = rtn_pack2_e4m3(v[4 * i], v[4 * i + 1]) | (rtn_pack2_e4m3(v[4 * i + 2], v[4 * i + 3]) << 16);
+            return round_pack16<FMT, RULE_RTN>(v, nullptr, qmax);
         }
     } else {
         uint32_t acc[EPL];
@@ -88,61 +81,59 @@ __device__ __forceinline__ uint4 round_pack_lane(const float* v, uint32_t acc0, 
                 acc[4 * g] = o.x; acc[4 * g + 1] = o.y; acc[4 * g + 2] = o.z; acc[4 * g + 3] = o.w;
             }
         }
+        // BF16 and FP16: the hardware stochastic-rounding converts.  Both take, per input, the leading bits of
+        // (threshold XOR sign mask); the two fields of a pair are assembled with byte permutes: the top halves of the two
+        // accumulators, XOR the two sign bytes replicated over their halves.
         if constexpr (FMT == FMT_BF16) {
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const uint32_t b0 = __float_as_uint(v[2 * i]), b1 = __float_as_uint(v[2 * i + 1]);
-                const uint32_t x0 = acc[2 * i] ^ (uint32_t)((int32_t)b0 >> 31);        // a negative value takes ~U
-                const uint32_t x1 = acc[2 * i + 1] ^ (uint32_t)((int32_t)b1 >> 31);
-                w[i] = sr_pack2_bf16(v[2 * i], v[2 * i + 1], x0, x1);
+                const uint32_t tops = __byte_perm(acc[2 * i], acc[2 * i + 1], 0x7632);
+                const uint32_t signs = sign_halves(v[2 * i], v[2 * i + 1]);
+                w[i] = sr_pack2_bf16_fields(v[2 * i], v[2 * i + 1], tops ^ signs);       // a negative value takes ~U
             }
         } else if constexpr (FMT == FMT_FP16) {
-            uint32_t unsure = 0;
+            float vmin0 = 3.0e38f, vmin1 = 3.0e38f;
+            uint32_t f[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const uint32_t b0 = __float_as_uint(v[2 * i]), b1 = __float_as_uint(v[2 * i + 1]);
-                const uint32_t x0 = acc[2 * i] ^ (uint32_t)((int32_t)b0 >> 31);
-                const uint32_t x1 = acc[2 * i + 1] ^ (uint32_t)((int32_t)b1 >> 31);
-                const uint32_t f = (x0 >> 19) | ((x1 >> 3) & 0x1FFF0000u);              // the leading 13 bits of each
-                const uint32_t f1 = f + 0x00010001u;
-                w[i] = sr_pack2_fp16(v[2 * i], v[2 * i + 1], f);
-                // the true addend lies in [f, f + 1): if the next field gives another code, or does not fit, decide exactly
-                unsure |= (w[i] ^ sr_pack2_fp16(v[2 * i], v[2 * i + 1], f1)) | (f1 & 0x20002000u);
+                const uint32_t tops = __byte_perm(acc[2 * i], acc[2 * i + 1], 0x7632);
+                const uint32_t signs = sign_halves(v[2 * i], v[2 * i + 1]);
+                f[i] = ((tops ^ signs) >> 3) & 0x1FFF1FFFu;                             // the leading 13 bits of each
+                if (i & 1) vmin1 = min3abs(vmin1, v[2 * i], v[2 * i + 1]);
+                else vmin0 = min3abs(vmin0, v[2 * i], v[2 * i + 1]);
             }
-            if (unsure) {
+            if (fminf(vmin0, vmin1) >= 0x1p-14f) {
+                // every target is in FP16's normal range: the 13 dropped bits are all carried by the field, one convert is exact
+#pragma unroll
+                for (int i = 0; i < 4; ++i) w[i] = sr_pack2_fp16(v[2 * i], v[2 * i + 1], f[i]);
+            } else {
+                // below 2^-14 the threshold has more leading bits than the field carries: fields f and f + 1 bracket the
+                // true addend, and where the two codes differ (or f + 1 does not fit) the lane decides exactly
+                uint32_t unsure = 0;
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    float r[2];
+                    const uint32_t f1 = f[i] + 0x00010001u;
+                    w[i] = sr_pack2_fp16(v[2 * i], v[2 * i + 1], f[i]);
+                    unsure |= (w[i] ^ sr_pack2_fp16(v[2 * i], v[2 * i + 1], f1)) | (f1 & 0x20002000u);
+                }
+                if (unsure) {
 #pragma unroll
-                    for (int j = 0; j < 2; ++j) {
-                        const float vv = v[2 * i + j];
-                        const float scale = dither_step_scale<10, -14, 24>(vv);
-                        const float q = floor_to_step(dithered_sum_rm(vv, acc[2 * i + j], scale), scale);
-                        // sign of v forced onto the result (it already has it unless it is zero)
-                        r[j] = __uint_as_float((__float_as_uint(q) & 0x7FFFFFFFu) | (__float_as_uint(vv) & 0x80000000u));
+                    for (int i = 0; i < 4; ++i) {
+                        float r[2];
+#pragma unroll
+                        for (int j = 0; j < 2; ++j) {
+                            const float vv = v[2 * i + j];
+                            const float scale = dither_step_scale<10, -14, 24>(vv);
+                            const float q = floor_to_step(dithered_sum_rm(vv, acc[2 * i + j], scale), scale);
+                            // sign of v forced onto the result (it already has it unless it is zero)
+                            r[j] = __uint_as_float((__float_as_uint(q) & 0x7FFFFFFFu) | (__float_as_uint(vv) & 0x80000000u));
+                        }
+                        w[i] = rtn_pack2_fp16(r[0], r[1]);   // exact: r is on the FP16 grid; saturates beyond 65504
                     }
-                    w[i] = rtn_pack2_fp16(r[0], r[1]);   // exact: r is on the FP16 grid; saturates beyond 65504
                 }
             }
-        } else if constexpr (FMT == FMT_INT) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-                w[i] = pack4_low_bytes(int_dither_biased(v[4 * i], acc[4 * i], qmax), int_dither_biased(v[4 * i + 1], acc[4 * i + 1], qmax),
-                                       int_dither_biased(v[4 * i + 2], acc[4 * i + 2], qmax), int_dither_biased(v[4 * i + 3], acc[4 * i + 3], qmax));
         } else {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                float r[4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const float vv = v[4 * i + j];
-                    const float scale = dither_step_scale<3, -6, 127>(vv);
-                    const float q = floor_to_step(dithered_sum_rm(vv, acc[4 * i + j], scale), scale);
-                    // sign of v forced onto the result (it already has it unless it is zero)
-                    r[j] = __uint_as_float((__float_as_uint(q) & 0x7FFFFFFFu) | (__float_as_uint(vv) & 0x80000000u));
-                }
-                w[i] = rtn_pack2_e4m3(r[0], r[1]) | (rtn_pack2_e4m3(r[2], r[3]) << 16);   // exact; saturates beyond 448
-            }
+            return round_pack16<FMT, RULE>(v, acc, qmax);
         }
     }
     return make_uint4(w[0], w[1], w[2], w[3]);
@@ -540,6 +531,7 @@ inline cudaError_t launch_update_one(const UpdateParams& p, cudaStream_t stream)
         if (aligned && q.B <= 65535u) {
 #define SSDQ_TILE_CASE(R)                                                                                          \
             if (q.P == nslot * (R)) {                                                                              \
+                note_kernel(1);                                                                                    \
                 if (extras) ssd_update_tile_kernel<FMT, RULE, LPR, R, true><<<tile_grid, kThreads, 0, stream>>>(q);  \
                 else ssd_update_tile_kernel<FMT, RULE, LPR, R, false><<<tile_grid, kThreads, 0, stream>>>(q);       \
                 return cudaGetLastError();                                                                         \
@@ -557,6 +549,7 @@ inline cudaError_t launch_update_one(const UpdateParams& p, cudaStream_t stream)
     q.items_per_cta = nslot / spi;
     q.rps = (q.P + spi - 1) / spi;
     const uint32_t grid = (q.n_items + q.items_per_cta - 1) / q.items_per_cta;
+    note_kernel(0);
     ssd_update_kernel<FMT, RULE, LPR, APS><<<grid, kThreads, 0, stream>>>(q);
     return cudaGetLastError();
 }

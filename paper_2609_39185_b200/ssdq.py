@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libssdq.so")
 EXPORTS = ("weyl_offsets_init", "ssdq_thresholds_materialize", "ssd_state_update", "quantize_store",
            "ssdq_dequantize", "ssd_decode_run", "ssd_decode_run_host", "ssd_replay_step", "ssd_decode_run_checkpointed",
            "ssd_decode_graph_create", "ssd_decode_graph_launch", "ssd_decode_graph_destroy", "ssdq_state_error_workspace_bytes", "ssdq_state_error",
-           "ssdq_state_error_static", "ssdq_readout_kl", "ssdq_last_error", "ssdq_launch_count")
+           "ssdq_state_error_static", "ssdq_readout_kl", "ssdq_copy", "ssdq_last_kernel", "ssdq_last_error", "ssdq_launch_count")
 
 _u32, _u64, _i32, _vp = ctypes.c_uint32, ctypes.c_uint64, ctypes.c_int32, ctypes.c_void_p
 
@@ -98,6 +98,10 @@ def lib() -> ctypes.CDLL:
         L.ssdq_state_error_static.argtypes = [_vp, _vp, _vp, _u32, _u32, _u32, _u32, ctypes.c_int, _u32, _vp, _vp, _vp]
         L.ssdq_readout_kl.restype = ctypes.c_int
         L.ssdq_readout_kl.argtypes = [_vp, _vp, _u32, _u32, _vp, _vp]
+        L.ssdq_copy.restype = ctypes.c_int
+        L.ssdq_copy.argtypes = [_vp, _vp, _u64, _vp]
+        L.ssdq_last_kernel.restype = ctypes.c_char_p
+        L.ssdq_last_kernel.argtypes = []
         L.ssdq_last_error.restype = ctypes.c_char_p
         L.ssdq_last_error.argtypes = []
         L.ssdq_launch_count.restype = _u64
@@ -289,6 +293,18 @@ class DecodeGraph:
             self.close()
         except Exception:
             pass
+
+
+def copy(src, dst):
+    """ssdq_copy: plain 128-bit copy of `src` into `dst` (same byte size) by the library's copy kernel -- the floor of
+    the timing protocol."""
+    nbytes = src.numel() * src.element_size()
+    assert nbytes == dst.numel() * dst.element_size()
+    _check(lib().ssdq_copy(_ptr(src), _ptr(dst), nbytes, _stream()))
+
+
+def last_kernel() -> str:
+    return lib().ssdq_last_kernel().decode()
 
 
 def launch_count() -> int:

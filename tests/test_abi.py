@@ -21,7 +21,7 @@ def lib():
 def declared_functions():
     text = open(os.path.join(ROOT, "include", "ssdq.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"^\s*(?:int|const char\*|uint64_t)\s+(\w+)\s*\(", text, flags=re.M)))
+    return sorted(set(re.findall(r"^\s*(?:ssdq_status|int|const char\*|uint64_t)\s+(\w+)\s*\(", text, flags=re.M)))
 
 
 def test_every_declared_symbol_is_exported(lib):
@@ -95,6 +95,43 @@ def test_quantize_and_driver_argument_checks(lib):
     s.ring = 2
     assert lib.ssd_decode_run(ctypes.byref(d), 1, 1, 4, ctypes.byref(s), None) == ssdq.ERR_NULL      # no inputs
     assert lib.ssd_decode_run(ctypes.byref(d), 1, 1, 0, ctypes.byref(s), None) == ssdq.OK            # zero steps
+
+
+def _step_inputs(ring=2, **over):
+    s = ssdq.StepInputs()
+    s.ring = ring
+    for name in ("x", "dt", "Bm", "Cm", "y"):
+        setattr(s, name, 0x40000)
+    s.stride_x = s.stride_dt = s.stride_B = s.stride_C = s.stride_y = s.stride_z = 64
+    for k, v in over.items():
+        setattr(s, k, v)
+    return s
+
+
+def test_a_misaligned_gate_is_rejected_by_every_driver(lib):
+    """z goes through the same pointer checks as x and y in the plain, the host-buffer, the checkpointed and the
+    graph driver; nothing is launched."""
+    d = _desc()
+    before = ssdq.launch_count()
+    bad = _step_inputs(z=0x40002)
+    assert lib.ssd_decode_run(ctypes.byref(d), 1, 1, 4, ctypes.byref(bad), None) == ssdq.ERR_ALIGN
+    good_host, bad_host = _step_inputs(z=0x40000), _step_inputs(z=0x40002)
+    good_staging, bad_staging = _step_inputs(z=0x50000), _step_inputs(z=0x50002)
+    assert lib.ssd_decode_run_host(ctypes.byref(d), 1, 1, 4, ctypes.byref(good_host), ctypes.byref(bad_staging), None) == ssdq.ERR_ALIGN
+    assert lib.ssd_decode_run_host(ctypes.byref(d), 1, 1, 4, ctypes.byref(bad_host), ctypes.byref(good_staging), None) == ssdq.ERR_ALIGN
+    work = (ctypes.c_void_p * 1)(0x60000)
+    assert lib.ssd_decode_run_checkpointed(ctypes.byref(d), work, 1, 2, 1, 4, ctypes.byref(bad), None) == ssdq.ERR_ALIGN
+    handle = ctypes.c_void_p()
+    assert lib.ssd_decode_graph_create(ctypes.byref(handle), ctypes.byref(d), 1, 2, ctypes.byref(bad), 0x70000) == ssdq.ERR_ALIGN
+    assert not handle.value and ssdq.launch_count() == before
+
+
+def test_copy_argument_checks(lib):
+    assert lib.ssdq_copy(None, 0x10000, 64, None) == ssdq.ERR_NULL
+    assert lib.ssdq_copy(0x10000, 0x20008, 64, None) == ssdq.ERR_ALIGN
+    assert lib.ssdq_copy(0x10000, 0x20000, 40, None) == ssdq.ERR_SHAPE
+    assert lib.ssdq_copy(0x10000, 0x20000, 0, None) == ssdq.OK
+    assert lib.ssdq_last_kernel() in (b"", b"ssd_update_kernel", b"ssd_update_tile_kernel", b"ssd_update_stream_kernel")
 
 
 def test_missing_library_fails_loudly(monkeypatch):

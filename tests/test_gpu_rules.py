@@ -139,3 +139,31 @@ def test_dequantize_matches_oracle(fmt):
     ssdq.dequantize(codes_to_dev(codes_h, fmt), to_dev(scales_h), fmt, out, scale_block=sb)
     want = oracle.dequantize(codes_h, scales_h, fmt, sb)
     assert np.array_equal(out.cpu().numpy().view(np.uint32), want.view(np.uint32))
+
+
+def test_exp_and_softplus_kernels_reproduce_the_known_answer_table(golden_dir):
+    """The frozen table guards both sides against a silent, matching change.  exp_spec: FP32-twin state h = 1, x = 0,
+    dt = 1, A = z, so the stored h' is a = exp_spec(z).  softplus_spec: h = 0, A = 0, x = B = 1 and in-kernel softplus,
+    so the stored h' is the step size softplus_spec(dt_raw)."""
+    from test_oracle_update import load_spec_kat
+    kat = load_spec_kat(golden_dir)
+    N = 16
+    for name in ("exp_spec", "softplus_spec"):
+        zin, zout = kat[name]
+        H = len(zin)
+        z = torch.from_numpy(zin.view(np.float32).copy()).cuda()
+        one = torch.ones((1, H), dtype=torch.float32, device="cuda")
+        y = torch.empty((1, H, 1), dtype=torch.float32, device="cuda")
+        if name == "exp_spec":
+            state = torch.ones((1, H, 1, N), dtype=torch.float32, device="cuda")
+            d = ssdq.make_desc(state, None, ssdq.FP32, A=z, D=None, rule=ssdq.RTN)
+            ssdq.ssd_state_update(d, 1, x=torch.zeros((1, H, 1), device="cuda"), dt=one, Bm=torch.ones((1, N), device="cuda"),
+                                  Cm=torch.zeros((1, N), device="cuda"), y=y)
+        else:
+            state = torch.zeros((1, H, 1, N), dtype=torch.float32, device="cuda")
+            d = ssdq.make_desc(state, None, ssdq.FP32, A=torch.zeros(H, device="cuda"), D=None, rule=ssdq.RTN, dt_softplus=True)
+            ssdq.ssd_state_update(d, 1, x=torch.ones((1, H, 1), device="cuda"), dt=z.view(1, H), Bm=torch.ones((1, N), device="cuda"),
+                                  Cm=torch.zeros((1, N), device="cuda"), y=y)
+        torch.cuda.synchronize()
+        got = state.cpu().numpy().view(np.uint32)[0, :, 0, :]
+        assert np.array_equal(got, np.repeat(zout[:, None], N, axis=1)), name

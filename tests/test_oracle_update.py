@@ -318,3 +318,27 @@ def test_replay_of_the_decomposed_step_reproduces_the_decode_step(fmt, rule):
         assert np.array_equal(st1.reshape(-1, N), st2)
         if sc1 is not None:
             assert np.array_equal(sc1, sc2)
+
+
+# ---- frozen known answers of the two fixed binary32 routines ---------------------------------------
+def load_spec_kat(golden_dir):
+    import os
+    table = {"exp_spec": [], "softplus_spec": []}
+    for line in open(os.path.join(golden_dir, "exp_softplus_kat.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        name, a, b = line.split()
+        table[name].append((int(a, 16), int(b, 16)))
+    return {k: (np.array([p[0] for p in v], np.uint32), np.array([p[1] for p in v], np.uint32)) for k, v in table.items()}
+
+
+def test_exp_and_softplus_reproduce_their_known_answer_table(golden_dir):
+    kat = load_spec_kat(golden_dir)
+    assert len(kat["exp_spec"][0]) >= 30 and len(kat["softplus_spec"][0]) >= 30
+    zin, zout = kat["exp_spec"]
+    assert np.array_equal(oracle.exp_spec(zin.view(np.float32)).view(np.uint32), zout)
+    xin, xout = kat["softplus_spec"]
+    assert np.array_equal(oracle.softplus_spec(xin.view(np.float32)).view(np.uint32), xout)
+    # the table is not self-referential noise: spot values against float64 (1 is exp(0); the rest within 3 ulp)
+    ref = np.exp(np.clip(zin.view(np.float32).astype(np.float64), -87.0, 88.0))
+    assert np.all(np.abs(zout.view(np.float32).astype(np.float64) - ref) <= 3 * np.spacing(ref.astype(np.float32)))
