@@ -73,9 +73,17 @@ ssdq_status check_layer(const ssdq_update_desc* d) {
     if (format_scaled(d->format)) {
         if (!d->scales) return fail(SSDQ_ERR_NULL, "E4M3 and INTb stores need a scale array");
         if (!aligned4(d->scales)) return fail(SSDQ_ERR_ALIGN, "scales are misaligned");
-        if (d->scale_block == (uint32_t)d->headdim * d->dstate && d->scale_block != d->dstate)
-            return fail(SSDQ_ERR_UNSUPPORTED, "one scale per head is not built; use scale_block 16 or dstate");
-        if (!(d->scale_block == 16 || d->scale_block == d->dstate)) return fail(SSDQ_ERR_SHAPE, "scale_block must be 16 or dstate");
+        const bool head_scale = d->scale_block == (uint32_t)d->headdim * d->dstate && d->scale_block != d->dstate;
+        if (head_scale) {
+            // one scale per (sequence, head): heads of (128 / lanes per row) * {2, 4, 8} rows, one decay per head, plain signature
+            const uint32_t lpr = d->dstate / 16u, rows = d->headdim * lpr;      // rows * 16 entries per lane set
+            const bool shape_ok = lpr >= 4 && lpr <= 16 && (rows == 128u * 2u || rows == 128u * 4u || rows == 128u * 8u);
+            if (!shape_ok || d->a_per_state || d->dt_bias || d->dt_softplus || d->z || d->ngroups > 1 || d->batch > 65535u)
+                return fail(SSDQ_ERR_UNSUPPORTED, "one scale per head (scale_block = headdim * dstate) is built for dstate 64..256, "
+                                                  "headdim * dstate / 2048 in {2, 4, 8}, one decay per head and the plain signature");
+        } else if (!(d->scale_block == 16 || d->scale_block == d->dstate)) {
+            return fail(SSDQ_ERR_SHAPE, "scale_block must be 16, dstate, or headdim * dstate");
+        }
     }
     if (d->rule == SSDQ_WEYL && d->format != SSDQ_FP32) {
         if (!(d->weyl.block == 16 || d->weyl.block == d->dstate)) return fail(SSDQ_ERR_SHAPE, "weyl.block must be 16 or dstate");
@@ -575,6 +583,7 @@ const char* ssdq_last_kernel(void) {
         case 0: return "ssd_update_kernel";
         case 1: return "ssd_update_tile_kernel";
         case 2: return "ssd_update_stream_kernel";
+        case 3: return "ssd_update_headscale_kernel";
         default: return "";
     }
 }

@@ -82,20 +82,22 @@ __device__ __forceinline__ uint4 round_pack_lane(const float* v, uint32_t acc0, 
             }
         }
         // BF16 and FP16: the hardware stochastic-rounding converts.  Both take, per input, the leading bits of
-        // (threshold XOR sign mask); the two fields of a pair are assembled with byte permutes: the top halves of the two
-        // accumulators, XOR the two sign bytes replicated over their halves.
+        // (threshold XOR sign mask): a negative value takes ~U.
         if constexpr (FMT == FMT_BF16) {
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const uint32_t tops = __byte_perm(acc[2 * i], acc[2 * i + 1], 0x7632);
-                const uint32_t signs = sign_halves(v[2 * i], v[2 * i + 1]);
-                w[i] = sr_pack2_bf16_fields(v[2 * i], v[2 * i + 1], tops ^ signs);       // a negative value takes ~U
+                const uint32_t b0 = __float_as_uint(v[2 * i]), b1 = __float_as_uint(v[2 * i + 1]);
+                const uint32_t x0 = acc[2 * i] ^ (uint32_t)((int32_t)b0 >> 31);
+                const uint32_t x1 = acc[2 * i + 1] ^ (uint32_t)((int32_t)b1 >> 31);
+                w[i] = sr_pack2_bf16_fields(v[2 * i], v[2 * i + 1], __byte_perm(x0, x1, 0x7632));     // the top halves
             }
         } else if constexpr (FMT == FMT_FP16) {
             float vmin0 = 3.0e38f, vmin1 = 3.0e38f;
             uint32_t f[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
+                // the two fields of a pair at once: the top halves of the two accumulators, XOR the two sign bytes
+                // replicated over their halves
                 const uint32_t tops = __byte_perm(acc[2 * i], acc[2 * i + 1], 0x7632);
                 const uint32_t signs = sign_halves(v[2 * i], v[2 * i + 1]);
                 f[i] = ((tops ^ signs) >> 3) & 0x1FFF1FFFu;                             // the leading 13 bits of each
@@ -512,11 +514,23 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
 template <int FMT, int RULE, int LPR>
 cudaError_t try_launch_stream(const UpdateParams& p, cudaStream_t stream, bool& launched);
 
+// The kernel of ssdq_headscale.cuh (one scale per (sequence, head)), for the shapes it covers.
+template <int FMT, int RULE, int LPR>
+cudaError_t try_launch_headscale(const UpdateParams& p, cudaStream_t stream, bool& launched);
+
 // Host-side launcher for one (format, rule): picks the lanes-per-row instantiation from N.
 template <int FMT, int RULE, int LPR, bool APS>
 inline cudaError_t launch_update_one(const UpdateParams& p, cudaStream_t stream) {
     UpdateParams q = p;
     const uint32_t nslot = kThreads / LPR;
+    if constexpr (Fmt<FMT>::kScaled) {
+        if (q.scale_block == q.P * q.N && q.scale_block != q.N) {       // one scale per head: its own kernel or nothing
+            bool launched = false;
+            cudaError_t e = cudaErrorInvalidValue;
+            if constexpr (!APS && LPR >= 4 && Fmt<FMT>::kBytes == 1) e = try_launch_headscale<FMT, RULE, LPR>(q, stream, launched);
+            return launched ? e : cudaErrorInvalidValue;
+        }
+    }
     if constexpr (!APS && LPR >= 4 && Fmt<FMT>::kScaled && Fmt<FMT>::kBytes == 1) {
         bool launched = false;
         const cudaError_t e = try_launch_stream<FMT, RULE, LPR>(q, stream, launched);

@@ -20,7 +20,7 @@ import numpy as np
 from . import workloads
 
 BINS = ((0.0, 10.0, "tau<10"), (10.0, 100.0, "tau10-100"), (100.0, 1000.0, "tau100-1000"), (1000.0, np.inf, "tau>=1000"))
-RULES = (("rtn", 0), ("sr", 1), ("weyl", 2))
+RULES = (("rtn", 0), ("sr", 1), ("weyl", 2), ("sr_hash", 3))
 
 
 def head_time_constants(cfg, A, mean_dt):
@@ -90,6 +90,7 @@ def main():
     ap.add_argument("--log-every", type=int, default=256)
     ap.add_argument("--batch", type=int, default=0)
     ap.add_argument("--format", default="", choices=["", "fp16", "bf16", "e4m3", "int8", "int7", "int6", "int4"])
+    ap.add_argument("--scale", default="", choices=["", "row", "block16", "head"], help="granularity of the FP32 scale of a scaled store")
     ap.add_argument("--out", default="")
     args = ap.parse_args()
     cfg = workloads.CONFIGS[args.config]
@@ -99,6 +100,8 @@ def main():
     if args.format:
         fmt = {v: k for k, v in workloads.FORMAT_NAMES.items()}[args.format]
         cfg = replace(cfg, fmt=fmt, scale_block=(cfg.scale_block or cfg.weyl_block) if fmt in workloads.SCALED_FORMATS else 0)
+    if args.scale and cfg.fmt in workloads.SCALED_FORMATS:
+        cfg = replace(cfg, scale_block={"row": cfg.dstate, "block16": 16, "head": cfg.headdim * cfg.dstate}[args.scale])
     out = open(args.out, "w") if args.out else None
 
     def emit(line):

@@ -156,3 +156,74 @@ def test_readout_kl_on_a_case_written_out_by_hand():
     assert oracle.readout_kl(y_q, y_ref)[0] == pytest.approx(0.5 * math.log(0.5 / (1 / 3)) + 0.5 * math.log(0.5 / (2 / 3)), rel=1e-12)
     # shape: any trailing dimensions are flattened per sequence
     assert oracle.readout_kl(y_ref.reshape(2, 3, 1), y_q.reshape(2, 3, 1)) == pytest.approx([want0, want1], rel=1e-12)
+
+
+# ---- one scale per (sequence, head): scale_block = P * N ---------------------------------------------------------
+@pytest.mark.parametrize("fmt", [E4M3, INT8])
+@pytest.mark.parametrize("rule", [RTN, WEYL, SR])
+def test_head_scale_step_against_an_element_by_element_restatement(fmt, rule):
+    """Section 2 "Low-precision storage" defines s = max|h| / top over a block; here the block is the whole head.  The
+    step is rebuilt from the pinned pieces: FP32 update, one scale from the head's maximum, v = h' * (1/s), threshold of
+    the flat index, Eq. 2, encode."""
+    rng = np.random.default_rng(300 + 10 * fmt + rule)
+    Bsz, H, P, N = 2, 3, 4, 32
+    sb = P * N
+    A = -np.exp(rng.uniform(-3, 1, H)).astype(f32)
+    state = rng.integers(-7, 8, (Bsz, H, P, N)).astype(np.int8).view(np.uint8) if fmt == INT8 else \
+        oracle.encode((rng.standard_normal((Bsz, H, P, N)) * 20).astype(f32), E4M3)
+    scales = rng.uniform(0.01, 0.2, Bsz * H).astype(f32)
+    x = rng.standard_normal((Bsz, H, P)).astype(f32)
+    dt = np.log1p(np.exp(rng.normal(-2, 0.5, (Bsz, H)))).astype(f32)
+    Bm = rng.standard_normal((Bsz, N)).astype(f32)
+    Cm = rng.standard_normal((Bsz, N)).astype(f32)
+    base, t = 5, 9
+    want_codes = np.zeros_like(state)
+    want_scales = np.zeros_like(scales)
+    want_y = np.zeros((Bsz, H, P))
+    for b in range(Bsz):
+        for h in range(H):
+            a = oracle.exp_spec(f32(dt[b, h] * A[h]))[0]
+            h_in = (oracle.decode(state[b, h], fmt) * scales[b * H + h]).astype(f32)
+            hp = np.zeros((P, N), f32)
+            for p in range(P):
+                dtx = f32(dt[b, h] * x[b, h, p])
+                for n in range(N):
+                    hp[p, n] = _fma32(a, h_in[p, n], f32(dtx * Bm[b, n]))
+                want_y[b, h, p] = float(np.dot(Cm[b].astype(np.float64), hp[p].astype(np.float64)))
+            s = max(f32(np.max(np.abs(hp)) / f32(TOP[fmt])), TINY)
+            want_scales[b * H + h] = s
+            rinv = f32(f32(1.0) / s)
+            for p in range(P):
+                for n in range(N):
+                    flat = ((((base + b) * H + h) * P + p) * N + n)
+                    U = oracle.threshold(rule, flat, t, layer=1, weyl_seed=0, weyl_block=16, sr_seed=77)
+                    want_codes[b, h, p, n] = oracle.encode(oracle.round_values(f32(hp[p, n] * rinv), U, fmt, rule), fmt)[0]
+    y = oracle.state_update(state, scales, fmt, sb, x, dt, A, Bm, Cm, None, rule, t, layer=1, weyl_block=16, sr_seed=77,
+                            batch_index_base=base)
+    assert np.array_equal(state, want_codes)
+    assert np.array_equal(scales, want_scales)
+    assert np.allclose(y, want_y, rtol=0, atol=1e-6 * np.max(np.abs(want_y)))
+    top_code = int(TOP[fmt]) if fmt == INT8 else 0x7E
+    mags = state.view(np.int8).astype(np.int32) if fmt == INT8 else (state & 0x7F).astype(np.int32)
+    assert np.all(np.abs(mags).reshape(Bsz * H, -1).max(axis=1) >= top_code - 1)       # the head's maximum lands on the top
+
+
+def test_head_scale_absorbs_a_shared_decay():
+    # one decay per head and no write: the single FP32 scale carries the decay and, under RTN, every code of the head stays
+    rng = np.random.default_rng(6)
+    Bsz, H, P, N = 1, 2, 4, 128
+    src = rng.standard_normal((Bsz * H, P * N)).astype(f32)
+    state = np.zeros((Bsz, H, P, N), np.uint8)
+    scales = np.zeros(Bsz * H, f32)
+    for i in range(Bsz * H):                     # quantise each head as one block of P * N entries
+        s = max(f32(np.max(np.abs(src[i])) / f32(448.0)), TINY)
+        scales[i] = s
+        state.reshape(Bsz * H, -1)[i] = oracle.round_encode((src[i] * f32(f32(1.0) / s)).astype(f32), None, E4M3, RTN)
+    before, s_before = state.copy(), scales.copy()
+    A = np.array([-0.5, -0.01], f32)
+    zero = np.zeros((Bsz, N), f32)
+    for t in range(1, 20):
+        oracle.state_update(state, scales, E4M3, P * N, np.zeros((Bsz, H, P), f32), np.full((Bsz, H), 0.1, f32), A, zero, zero,
+                            None, RTN, t, weyl_block=128)
+    assert np.array_equal(state, before)
+    assert np.allclose(scales / s_before, np.exp(0.1 * A.astype(np.float64)) ** 19, rtol=1e-5)
