@@ -167,3 +167,53 @@ def test_exp_and_softplus_kernels_reproduce_the_known_answer_table(golden_dir):
         torch.cuda.synchronize()
         got = state.cpu().numpy().view(np.uint32)[0, :, 0, :]
         assert np.array_equal(got, np.repeat(zout[:, None], N, axis=1)), name
+
+
+def _contraction_sensitive_tie():
+    """(amax, h, k_even): the block scale s = amax / 127 and h are such that RN(h * RN(1/s)) is exactly k + 1/2 while the
+    exact product is not: a multiply that is fused into the rounding add would round to the nearer integer instead of
+    the even one.  Checked here in exact arithmetic before it is used."""
+    f32 = np.float32
+    s = np.uint32(1021728416).view(f32)
+    h = np.uint32(3196633967).view(f32)
+    amax = None
+    for cand in np.nextafter(f32(s * f32(127.0)), [f32(0), f32(1e9)], dtype=f32).tolist() + [float(f32(s * f32(127.0)))]:
+        if f32(f32(cand) / f32(127.0)) == s:
+            amax = f32(cand)
+    assert amax is not None
+    rinv = f32(f32(1.0) / s)
+    v = f32(h * rinv)
+    exact = Fraction(float(h)) * Fraction(float(rinv))
+    assert float(v) == -9.5 and exact != Fraction(-19, 2) and exact > Fraction(-19, 2)      # nearest of the exact product: -9; ties-to-even of v: -10
+    return amax, h, -10
+
+
+def test_int8_rtn_tie_is_not_moved_by_a_fused_multiply_add():
+    """v = h' * (1/s) is rounded BEFORE it is rounded onto the integer grid (two operations); every kernel that writes
+    INT8 codes must keep the tie: quantize_store, the persistent kernel, the per-head-scale kernel and the generic one."""
+    amax, h, want = _contraction_sensitive_tie()
+    N = 128
+    row = np.zeros(N, np.float32)
+    row[0], row[1], row[17] = amax, h, h
+    want_row = oracle.quantize_store(row.reshape(1, N), oracle.INT8, oracle.RTN, 1, scale_block=N)[0].view(np.int8)[0]
+    assert want_row[1] == want and want_row[17] == want and want_row[0] == 127
+    # quantize_store
+    src = np.tile(row, (64, 1))
+    codes = torch.zeros((64, N), dtype=torch.uint8, device="cuda")
+    scales = torch.zeros((64, 1), dtype=torch.float32, device="cuda")
+    ssdq.quantize_store(to_dev(src), codes, scales, ssdq.INT8, ssdq.RTN, 1, scale_block=N)
+    assert np.array_equal(codes.cpu().numpy().view(np.int8), np.tile(want_row, (64, 1)))
+    # the decode step: zero state, A = 0 (a = 1), dt = x = 1, so h' = B[n] on every row
+    for shape, sb, kernel in (((2, 3, 64, N), N, "ssd_update_stream_kernel"), ((2, 3, 64, N), 64 * N, "ssd_update_headscale_kernel"),
+                              ((2, 3, 5, N), N, "ssd_update_kernel"), ((2, 3, 32, N), N, "ssd_update_tile_kernel")):
+        B, H, P, _ = shape
+        state = torch.zeros(shape, dtype=torch.uint8, device="cuda")
+        sc = torch.full((B * H * P * N // sb,), float(np.finfo(np.float32).tiny), dtype=torch.float32, device="cuda")
+        d = ssdq.make_desc(state, sc, ssdq.INT8, A=torch.zeros(H, device="cuda"), D=None, rule=ssdq.RTN, scale_block=sb)
+        ssdq.ssd_state_update(d, 1, x=torch.ones((B, H, P), device="cuda"), dt=torch.ones((B, H), device="cuda"),
+                              Bm=to_dev(np.tile(row, (B, 1))), Cm=torch.zeros((B, N), device="cuda"),
+                              y=torch.empty((B, H, P), device="cuda"))
+        torch.cuda.synchronize()
+        assert ssdq.last_kernel() == kernel
+        got = state.cpu().numpy().view(np.int8).reshape(-1, N)
+        assert np.array_equal(got, np.tile(want_row, (len(got), 1))), kernel
