@@ -584,6 +584,7 @@ const char* ssdq_last_kernel(void) {
         case 1: return "ssd_update_tile_kernel";
         case 2: return "ssd_update_stream_kernel";
         case 3: return "ssd_update_headscale_kernel";
+        case 4: return "ssd_update_mamba1_kernel";
         default: return "";
     }
 }

@@ -514,6 +514,10 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
 template <int FMT, int RULE, int LPR>
 cudaError_t try_launch_stream(const UpdateParams& p, cudaStream_t stream, bool& launched);
 
+// The kernel of ssdq_mamba1.cuh (N = 16, headdim 1, one decay per state), for the calls it covers.
+template <int FMT, int RULE>
+cudaError_t try_launch_mamba1(const UpdateParams& p, cudaStream_t stream, bool& launched);
+
 // The kernel of ssdq_headscale.cuh (one scale per (sequence, head)), for the shapes it covers.
 template <int FMT, int RULE, int LPR>
 cudaError_t try_launch_headscale(const UpdateParams& p, cudaStream_t stream, bool& launched);
@@ -523,6 +527,11 @@ template <int FMT, int RULE, int LPR, bool APS>
 inline cudaError_t launch_update_one(const UpdateParams& p, cudaStream_t stream) {
     UpdateParams q = p;
     const uint32_t nslot = kThreads / LPR;
+    if constexpr (APS && FMT != FMT_FP32 && LPR * Fmt<FMT>::kEpl == 16) {
+        bool launched = false;
+        const cudaError_t e = try_launch_mamba1<FMT, RULE>(q, stream, launched);
+        if (launched || e != cudaSuccess) return e;
+    }
     if constexpr (Fmt<FMT>::kScaled) {
         if (q.scale_block == q.P * q.N && q.scale_block != q.N) {       // one scale per head: its own kernel or nothing
             bool launched = false;

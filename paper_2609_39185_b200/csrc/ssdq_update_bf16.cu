@@ -1,5 +1,6 @@
 // Instantiations of the fused decode-step kernel for the bf16 state store.
 #include "ssdq_update.cuh"
+#include "ssdq_mamba1.cuh"
 
 namespace ssdq {
 cudaError_t launch_update_bf16(const UpdateParams& p, int rule, bool a_per_state, cudaStream_t s) {

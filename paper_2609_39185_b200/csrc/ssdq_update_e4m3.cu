@@ -1,5 +1,6 @@
 // Instantiations of the fused decode-step kernel for the e4m3 state store.
 #include "ssdq_stream.cuh"
+#include "ssdq_mamba1.cuh"
 #include "ssdq_headscale.cuh"
 
 namespace ssdq {

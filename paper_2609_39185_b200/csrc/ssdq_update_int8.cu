@@ -1,6 +1,7 @@
 // Instantiations of the fused decode-step kernel for the symmetric block-absmax integer stores (INT8/7/6/4 in an
 // int8 container; q_max is a run-time parameter).
 #include "ssdq_stream.cuh"
+#include "ssdq_mamba1.cuh"
 #include "ssdq_headscale.cuh"
 
 namespace ssdq {
