@@ -100,7 +100,7 @@ __device__ __forceinline__ uint4 round_pack_lane(const float* v, uint32_t acc0, 
                 // replicated over their halves
                 const uint32_t tops = __byte_perm(acc[2 * i], acc[2 * i + 1], 0x7632);
                 const uint32_t signs = sign_halves(v[2 * i], v[2 * i + 1]);
-                f[i] = ((tops ^ signs) >> 3) & 0x1FFF1FFFu;                             // the leading 13 bits of each
+                f[i] = (tops ^ signs) >> 3;        // the leading 13 bits of each in [12:0] and [28:16]; the convert ignores bits [15:13]
                 if (i & 1) vmin1 = min3abs(vmin1, v[2 * i], v[2 * i + 1]);
                 else vmin0 = min3abs(vmin0, v[2 * i], v[2 * i + 1]);
             }
@@ -114,7 +114,7 @@ __device__ __forceinline__ uint4 round_pack_lane(const float* v, uint32_t acc0, 
                 uint32_t unsure = 0;
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const uint32_t f1 = f[i] + 0x00010001u;
+                    const uint32_t f1 = (f[i] & 0x1FFF1FFFu) + 0x00010001u;
                     w[i] = sr_pack2_fp16(v[2 * i], v[2 * i + 1], f[i]);
                     unsure |= (w[i] ^ sr_pack2_fp16(v[2 * i], v[2 * i + 1], f1)) | (f1 & 0x20002000u);
                 }
@@ -426,7 +426,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
 #pragma unroll
         for (int k = 0; k < RPS; ++k) sc[k] = row_scale ? p.scales[row_first + k] : p.scales[(row_first + k) * (N / 16) + lis];
     }
-    float Bv[EPL], Cv[EPL];
+    f32x2 B2[EPL / 2], C2[EPL / 2];
     {
         const size_t grp = (!EXTRAS || p.ngroups == 1) ? (size_t)b : (size_t)b * p.ngroups + h / p.heads_per_group;
         const float4* Bp = reinterpret_cast<const float4*>(p.Bm + grp * N + n0);
@@ -434,8 +434,8 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
 #pragma unroll
         for (int i = 0; i < EPL / 4; ++i) {
             const float4 bb = __ldg(Bp + i), cc = __ldg(Cp + i);
-            Bv[4 * i] = bb.x; Bv[4 * i + 1] = bb.y; Bv[4 * i + 2] = bb.z; Bv[4 * i + 3] = bb.w;
-            Cv[4 * i] = cc.x; Cv[4 * i + 1] = cc.y; Cv[4 * i + 2] = cc.z; Cv[4 * i + 3] = cc.w;
+            B2[2 * i] = pack2(bb.x, bb.y); B2[2 * i + 1] = pack2(bb.z, bb.w);
+            C2[2 * i] = pack2(cc.x, cc.y); C2[2 * i + 1] = pack2(cc.z, cc.w);
         }
     }
     float dtv = __ldg(p.dt + item);
@@ -450,6 +450,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
     for (int g4 = 0; g4 < RPS / GRP; ++g4)
         gate[g4] = (EXTRAS && p.z && y_writer) ? __ldg(p.z + row_first + g4 * GRP + lis / (LPR / GRP)) : 0.0f;
     const float a = exp_spec(__fmul_rn(dtv, __ldg(p.A + h)));
+    const f32x2 a2 = pack2(a, a);
     const float Dl = (p.D && lis == 0) ? __ldg(p.D + h) : 0.0f;     // the skip term enters the dot on one lane
 
     LaneThreshold<FMT, RULE, LPR> thr;
@@ -471,19 +472,27 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
             float hv[EPL];
             cp_async_wait_rows<RPS>(k);                       // rows 0..k have landed
             unpack_lane<FMT>(tile[k][threadIdx.x], hv);
+            // Eq. 1 and the partial readout, two entries per instruction (packed binary32: the same operations and roundings)
             const float dtx = __fmul_rn(dtv, xv[k]);
-            float dot = __fmul_rn(Dl, xv[k]);
+            const f32x2 dtx2 = pack2(dtx, dtx);
+            f32x2 dot2 = pack2(__fmul_rn(Dl, xv[k]), 0.0f);
             float amax = 0.0f;
+            f32x2 hn2[EPL / 2];
 #pragma unroll
-            for (int j = 0; j < EPL; ++j) {
-                float hin = hv[j];
-                if constexpr (Fmt<FMT>::kScaled) hin = __fmul_rn(hin, sc[k]);
-                const float hn = __fmaf_rn(a, hin, __fmul_rn(dtx, Bv[j]));
-                hv[j] = hn;
-                dot = __fmaf_rn(Cv[j], hn, dot);
-                if constexpr (Fmt<FMT>::kScaled) amax = fmaxf(amax, fabsf(hn));
+            for (int i = 0; i < EPL / 2; ++i) {
+                f32x2 hin = pack2(hv[2 * i], hv[2 * i + 1]);
+                if constexpr (Fmt<FMT>::kScaled) hin = mul2_rn(hin, pack2(sc[k], sc[k]));
+                const f32x2 hn = fma2_rn(a2, hin, mul2_rn(dtx2, B2[i]));
+                hn2[i] = hn;
+                dot2 = fma2_rn(C2[i], hn, dot2);
+                unpack2(hn, hv[2 * i], hv[2 * i + 1]);
+                if constexpr (Fmt<FMT>::kScaled) amax = max3abs(amax, hv[2 * i], hv[2 * i + 1]);
             }
-            dots[u] = dot;
+            {
+                float d0, d1;
+                unpack2(dot2, d0, d1);
+                dots[u] = __fadd_rn(d0, d1);
+            }
             if constexpr (Fmt<FMT>::kScaled) {
                 if (row_scale) {
 #pragma unroll
@@ -491,8 +500,9 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
                 }
                 const float s = fmaxf(__fdiv_rn(amax, p.scale_top), 1.17549435e-38f);
                 const float rinv = __frcp_rn(s);
+                const f32x2 rinv2 = pack2(rinv, rinv);
 #pragma unroll
-                for (int j = 0; j < EPL; ++j) hv[j] = __fmul_rn(hv[j], rinv);
+                for (int i = 0; i < EPL / 2; ++i) unpack2(mul2_rn(hn2[i], rinv2), hv[2 * i], hv[2 * i + 1]);
                 if (row_scale) { if (lis == 0) p.scales[row_first + k] = s; }
                 else p.scales[(row_first + k) * (N / 16) + lis] = s;
             }
