@@ -15,15 +15,15 @@ namespace ssdq {
 // adding and subtracting 1.5 * 2^23 with SCALAR adds (a packed add after the packed multiply would be contracted into a
 // fused multiply-add by the assembler and could move k); the integer k then sits in the low bits of the sum.
 __device__ __forceinline__ f32x2 exp_spec2(f32x2 z2) {
-    float z0, z1;
-    unpack2(z2, z0, z1);
-    z0 = fminf(fmaxf(z0, -87.0f), 88.0f);
-    z1 = fminf(fmaxf(z1, -87.0f), 88.0f);
-    z2 = pack2(z0, z1);
+    {
+        float z0, z1;
+        unpack2(z2, z0, z1);
+        z2 = pack2(fminf(fmaxf(z0, -87.0f), 88.0f), fminf(fmaxf(z1, -87.0f), 88.0f));
+    }
     float t0, t1;
     unpack2(mul2_rn(z2, pack2(0x1.715476p+0f, 0x1.715476p+0f)), t0, t1);
     const float m0 = __fadd_rn(t0, 12582912.0f), m1 = __fadd_rn(t1, 12582912.0f);       // nearest-even integer, |t| < 2^22
-    const f32x2 k2 = pack2(__fadd_rn(m0, -12582912.0f), __fadd_rn(m1, -12582912.0f));
+    const f32x2 k2 = add2_rn(pack2(m0, m1), pack2(-12582912.0f, -12582912.0f));         // exact; its inputs are sums, not products
     f32x2 r = fma2_rn(k2, pack2(-0x1.62e400p-1f, -0x1.62e400p-1f), z2);
     r = fma2_rn(k2, pack2(-0x1.7f7d1cp-20f, -0x1.7f7d1cp-20f), r);
     f32x2 p = pack2(0x1.a01a02p-13f, 0x1.a01a02p-13f);
