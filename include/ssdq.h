@@ -246,9 +246,20 @@ ssdq_status ssdq_readout_kl(const float* y_ref, const float* y_q, uint32_t batch
  * of the same buffers launched the same way (the "copy" column of Table 11, Section 6.5 "Cost"). */
 ssdq_status ssdq_copy(const void* src, void* dst, uint64_t bytes, void* stream);
 
+/* Bounds-checking build.  A library compiled with -DSSDQ_DEBUG (python -m paper_2609_39185_b200.build --debug gives
+ * libssdq_debug.so) makes every fused-update kernel compare the index ranges it derives with the extents implied by the
+ * descriptor before touching memory; a lane that would step outside records the first violation and skips its accesses
+ * (nothing traps, the context stays usable).  This call waits for earlier work on the device and copies the four status
+ * words to out4 (HOST): code (0 = no violation; 1 state, 2 x/y rows, 3 scales, 4 dt items, 5 B/C), offending index low and
+ * high word, block index; reset != 0 clears them afterwards.  In a release build it returns SSDQ_ERR_UNSUPPORTED.
+ * It stands in for a memory checker on systems where none can be run. */
+ssdq_status ssdq_debug_status(uint32_t* out4, int reset);
+
 /* Name of the kernel family that the last fused-update launch issued from this thread used:
  * "ssd_update_stream_kernel" (persistent, one-byte block-scaled stores on head-shaped tiles),
- * "ssd_update_tile_kernel" (one CTA per head) or "ssd_update_kernel" (any shape); "" before the first launch.
+ * "ssd_update_tile_kernel" (one CTA per head), "ssd_update_headscale_kernel" (one scale per head),
+ * "ssd_update_mamba1_kernel" (dstate 16, headdim 1, one decay per state) or "ssd_update_kernel" (any shape); "" before
+ * the first launch.
  * For benchmark records. */
 const char* ssdq_last_kernel(void);
 

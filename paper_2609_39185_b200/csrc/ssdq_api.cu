@@ -99,6 +99,23 @@ ssdq_status check_step_ptrs(const float* x, const float* dt, const float* Bm, co
     return SSDQ_OK;
 }
 
+#ifdef SSDQ_DEBUG
+// The status words of the bounds-checking build: code of the first violation (0 = none), the offending index (low, high)
+// and the block that saw it.
+__device__ uint32_t g_debug_status[4];
+uint32_t* debug_status_address() {
+    static uint32_t* cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!cached[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_debug_status) != cudaSuccess) return nullptr;
+        cached[dev] = static_cast<uint32_t*>(ptr);
+    }
+    return cached[dev];
+}
+#endif
+
 ssdq::UpdateParams make_params(const ssdq_update_desc* d, uint32_t step_t) {
     ssdq::UpdateParams p{};
     p.state = d->state; p.scales = d->scales;
@@ -114,6 +131,18 @@ ssdq::UpdateParams make_params(const ssdq_update_desc* d, uint32_t step_t) {
     p.step_t = step_t; p.layer = d->layer; p.batch_base = d->batch_index_base;
     p.weyl = weyl_const(d->weyl);
     p.sr_seed = d->sr_seed;
+#ifdef SSDQ_DEBUG
+    {
+        const uint64_t rows = (uint64_t)d->batch * d->nheads * d->headdim, entries = rows * d->dstate;
+        const uint64_t bytes = d->format == SSDQ_FP32 ? 4u : (d->format == SSDQ_FP16 || d->format == SSDQ_BF16) ? 2u : 1u;
+        p.dbg.status = debug_status_address();
+        p.dbg.state_vecs = entries * bytes / 16u;
+        p.dbg.rows = rows;
+        p.dbg.scales = format_scaled(d->format) && d->scale_block ? entries / d->scale_block : 0u;
+        p.dbg.items = (uint64_t)d->batch * d->nheads;
+        p.dbg.bc_floats = (uint64_t)d->batch * p.ngroups * d->dstate;
+    }
+#endif
     return p;
 }
 
@@ -302,6 +331,10 @@ ssdq_status ssd_decode_run_checkpointed(const ssdq_update_desc* layers, float* c
             // the update itself runs on the FP32 working state, unrounded
             ssdq::UpdateParams p = make_params(&d, t);
             p.state = work_fp32[l]; p.scales = nullptr; p.scale_block = 0;
+#ifdef SSDQ_DEBUG
+            p.dbg.state_vecs = (uint64_t)d.batch * d.nheads * d.headdim * d.dstate / 4u;      // binary32 working state
+            p.dbg.scales = 0;
+#endif
             p.x = in->x + k * in->stride_x;
             p.dt = in->dt + k * in->stride_dt;
             p.Bm = in->Bm + k * in->stride_B;
@@ -576,6 +609,21 @@ ssdq_status ssdq_copy(const void* src, void* dst, uint64_t bytes, void* stream) 
     if (bytes % 16 != 0) return fail(SSDQ_ERR_SHAPE, "bytes must be a multiple of 16");
     if (!aligned16(src) || !aligned16(dst)) return fail(SSDQ_ERR_ALIGN, "src and dst must be 16-byte aligned");
     return cuda_result(ssdq::launch_copy(src, dst, bytes, static_cast<cudaStream_t>(stream)), "copy kernel");
+}
+
+ssdq_status ssdq_debug_status(uint32_t* out4, int reset) {
+#ifdef SSDQ_DEBUG
+    if (!out4) return fail(SSDQ_ERR_NULL, "out4 is NULL");
+    uint32_t* dev = debug_status_address();
+    if (!dev) return fail(SSDQ_ERR_CUDA, "no address for the debug status words");
+    cudaError_t e = cudaMemcpy(out4, dev, 4 * sizeof(uint32_t), cudaMemcpyDeviceToHost);      // synchronises with earlier work
+    if (e == cudaSuccess && reset) e = cudaMemset(dev, 0, 4 * sizeof(uint32_t));
+    if (e != cudaSuccess) return fail(SSDQ_ERR_CUDA, "debug status: %s", cudaGetErrorString(e));
+    return SSDQ_OK;
+#else
+    (void)out4; (void)reset;
+    return fail(SSDQ_ERR_UNSUPPORTED, "not a bounds-checking build (compile with -DSSDQ_DEBUG)");
+#endif
 }
 
 const char* ssdq_last_kernel(void) {

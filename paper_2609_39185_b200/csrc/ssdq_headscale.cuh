@@ -32,30 +32,35 @@ __global__ void __launch_bounds__(kThreads) ssd_update_headscale_kernel(const Up
     __shared__ uint4 tile[RPS][kThreads];
     __shared__ float warp_max[kThreads / 32];
     uint4* sp = reinterpret_cast<uint4*>(p.state) + row_first * LPR + lis;
+    // debug builds: everything this lane will touch, checked once (a lane that fails keeps running but accesses nothing)
+    const bool mem_ok = SSDQ_RANGE_OK(p, DBG_STATE, row_first * LPR + lis, (RPS - 1) * LPR + 1, state_vecs) &&
+                        SSDQ_RANGE_OK(p, DBG_ROWS, row_first, RPS, rows) && SSDQ_RANGE_OK(p, DBG_ITEMS, item, 1, items) &&
+                        SSDQ_RANGE_OK(p, DBG_SCALES, item, 1, scales) && SSDQ_RANGE_OK(p, DBG_BC, (size_t)b * N + n0, EPL, bc_floats);
 #pragma unroll
     for (int k = 0; k < RPS; ++k) {
         const uint32_t dst = (uint32_t)__cvta_generic_to_shared(&tile[k][threadIdx.x]);
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n cp.async.commit_group;" ::"r"(dst), "l"(sp + k * LPR) : "memory");
+        if (mem_ok) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n cp.async.commit_group;" ::"r"(dst), "l"(sp + k * LPR) : "memory");
     }
     float xv[RPS];
 #pragma unroll
     for (int k = 0; k < RPS / 2; ++k) {
-        const float2 x2 = __ldg(reinterpret_cast<const float2*>(p.x + row_first) + k);
+        const float2 x2 = mem_ok ? __ldg(reinterpret_cast<const float2*>(p.x + row_first) + k) : make_float2(0.0f, 0.0f);
         xv[2 * k] = x2.x; xv[2 * k + 1] = x2.y;
     }
-    const float sc_old = p.scales[item];
+    const float sc_old = mem_ok ? p.scales[item] : 0.0f;
     f32x2 B2[EPL / 2], C2[EPL / 2];
     {
         const float4* Bp = reinterpret_cast<const float4*>(p.Bm + (size_t)b * N + n0);
         const float4* Cp = reinterpret_cast<const float4*>(p.Cm + (size_t)b * N + n0);
 #pragma unroll
         for (int i = 0; i < EPL / 4; ++i) {
-            const float4 bb = __ldg(Bp + i), cc = __ldg(Cp + i);
+            const float4 zero4 = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            const float4 bb = mem_ok ? __ldg(Bp + i) : zero4, cc = mem_ok ? __ldg(Cp + i) : zero4;
             B2[2 * i] = pack2(bb.x, bb.y); B2[2 * i + 1] = pack2(bb.z, bb.w);
             C2[2 * i] = pack2(cc.x, cc.y); C2[2 * i + 1] = pack2(cc.z, cc.w);
         }
     }
-    const float dtv = __ldg(p.dt + item);
+    const float dtv = mem_ok ? __ldg(p.dt + item) : 0.0f;
     const float a = exp_spec(__fmul_rn(dtv, __ldg(p.A + h)));
     const float Dl = (p.D && lis == 0) ? __ldg(p.D + h) : 0.0f;
     const f32x2 a2 = pack2(a, a), sc2 = pack2(sc_old, sc_old);
@@ -100,7 +105,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_headscale_kernel(const Up
         float tot;
         if constexpr (GRP == 4) tot = reduce4_over_slot<LPR>(dots[0], dots[1], dots[2], dots[3], lis);
         else tot = reduce2_over_slot<LPR>(dots[0], dots[1], lis);
-        if (y_writer) p.y[row_first + g * GRP + lis / (LPR / GRP)] = tot;
+        if (y_writer && mem_ok) p.y[row_first + g * GRP + lis / (LPR / GRP)] = tot;
     }
     // the head's maximum: warp shuffle, then across the warps through shared memory
 #pragma unroll
@@ -112,7 +117,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_headscale_kernel(const Up
     const float s = fmaxf(__fdiv_rn(amax, p.scale_top), 1.17549435e-38f);
     const float rinv = __frcp_rn(s);
     const f32x2 rinv2 = pack2(rinv, rinv);
-    if (threadIdx.x == 0) p.scales[item] = s;
+    if (threadIdx.x == 0 && mem_ok) p.scales[item] = s;
 
     // pass 2: scale, thresholds, Eq. 2, store
     LaneThreshold<FMT, RULE, LPR> thr;
@@ -130,8 +135,9 @@ __global__ void __launch_bounds__(kThreads) ssd_update_headscale_kernel(const Up
 #pragma unroll
         for (int i = 0; i < EPL / 2; ++i) unpack2(mul2_rn(hn[k][i], rinv2), v[2 * i], v[2 * i + 1]);
         if constexpr (RULE == RULE_SR_HASH) acc_row = thr.hash_key0(grow_first + k, hash_base, key1);
-        sp[k * LPR] = round_pack_lane<FMT, RULE>(v, acc_row, p.weyl.mul_col, (uint32_t)grp_row, (uint32_t)(grp_row >> 32), step_t,
+        const uint4 packed = round_pack_lane<FMT, RULE>(v, acc_row, p.weyl.mul_col, (uint32_t)grp_row, (uint32_t)(grp_row >> 32), step_t,
                                                  p.layer, key0, key1, p.scale_top);
+        if (mem_ok) sp[k * LPR] = packed;
         if constexpr (RULE == RULE_WEYL) acc_row += thr.row_mul;
         if constexpr (RULE == RULE_SR) grp_row += N / 4;
     }

@@ -6,6 +6,20 @@
 
 namespace ssdq {
 
+// Debug builds (-DSSDQ_DEBUG) carry the extents of the caller's buffers into every update kernel: each lane checks the
+// index ranges it derives against them before it touches memory, records the first violation in a status word and skips
+// its accesses (no trap), and the C ABI reports the word (ssdq_debug_status).  Release builds compile none of this.
+#ifdef SSDQ_DEBUG
+struct DebugBounds {
+    uint32_t* status;        // [4] device words: code, index low, index high, blockIdx.x of the first violation
+    uint64_t state_vecs;     // 16-byte vectors in the state
+    uint64_t rows;           // B * H * P: extent of x, y (and z)
+    uint64_t scales;         // FP32 scales
+    uint64_t items;          // B * H: extent of dt
+    uint64_t bc_floats;      // B * G * N: extent of Bm, Cm
+};
+#endif
+
 // Kernel parameters of one fused update launch (copied by value into constant memory at launch).
 struct UpdateParams {
     void* state;
@@ -36,6 +50,9 @@ struct UpdateParams {
     uint32_t rps;            // rows per slot
     WeylConst weyl;
     uint64_t sr_seed;
+#ifdef SSDQ_DEBUG
+    DebugBounds dbg;
+#endif
 };
 
 // Parameters of quantize_store / replay / dequantize / thresholds.

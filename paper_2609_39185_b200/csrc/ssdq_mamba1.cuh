@@ -72,6 +72,11 @@ __global__ void __launch_bounds__(kThreads) ssd_update_mamba1_kernel(const Updat
         const uint64_t row = (uint64_t)b * p.H + d;
         const uint64_t grow = row + (uint64_t)p.batch_base * p.H;
         uint4* sp = reinterpret_cast<uint4*>(p.state) + row * CH;
+        // debug builds: the row's vectors, its x / y / dt elements, its scale and the sequence's B and C
+        bool mem_ok = SSDQ_RANGE_OK(p, DBG_STATE, row * CH, CH, state_vecs) && SSDQ_RANGE_OK(p, DBG_ROWS, row, 1, rows) &&
+                      SSDQ_RANGE_OK(p, DBG_ITEMS, row, 1, items) && SSDQ_RANGE_OK(p, DBG_BC, (size_t)b * N, N, bc_floats);
+        if constexpr (Fmt<FMT>::kScaled) mem_ok = mem_ok && SSDQ_RANGE_OK(p, DBG_SCALES, row, 1, scales);
+        if (!mem_ok) continue;          // a lane on its own: nothing below involves another thread
         uint4 raw[CH];
 #pragma unroll
         for (int c = 0; c < CH; ++c) raw[c] = sp[c];

@@ -94,6 +94,11 @@ __global__ void __launch_bounds__(kThreads, SSDQ_STREAM_MINB) ssd_update_stream_
     float* c_y = p.y + row0 + lis / (LPR / 4);
 
     auto issue = [&](uint32_t stage) {
+        // debug builds: the item's codes, x and scales must lie inside the caller's buffers (else nothing is copied)
+        const uint64_t frow = (uint64_t)(f_x - p.x);
+        bool mem_ok = SSDQ_RANGE_OK(p, DBG_STATE, frow * LPR + lis, (RPS - 1) * LPR + 1, state_vecs) && SSDQ_RANGE_OK(p, DBG_ROWS, frow, RPS, rows) &&
+                      SSDQ_RANGE_OK(p, DBG_SCALES, frow * SPR + (ROW_SCALE ? 0u : lis), (RPS - 1) * SPR + 1, scales);
+        if (mem_ok) {
 #pragma unroll
         for (int k = 0; k < RPS; ++k) cp_async16(tile_s + stage * kTileStage + k * (kThreads * 16u), f_codes + k * LPR);
 #pragma unroll
@@ -106,6 +111,7 @@ __global__ void __launch_bounds__(kThreads, SSDQ_STREAM_MINB) ssd_update_stream_
 #pragma unroll
                 for (int j = 0; j < 4; ++j) cp_async4_ca(sdst + 4 * j, f_sc + (4 * k4 + j) * SPR);
             }
+        }
         }
         f_codes += ROWS * LPR;
         f_x += ROWS;
@@ -137,9 +143,11 @@ __global__ void __launch_bounds__(kThreads, SSDQ_STREAM_MINB) ssd_update_stream_
       {
         const float4* Bp = reinterpret_cast<const float4*>(p.Bm + (size_t)b * N + n0);
         const float4* Cp = reinterpret_cast<const float4*>(p.Cm + (size_t)b * N + n0);
+        const bool bc_ok = SSDQ_RANGE_OK(p, DBG_BC, (size_t)b * N + n0, EPL, bc_floats);
 #pragma unroll
         for (int i = 0; i < EPL / 4; ++i) {
-            const float4 bb = __ldg(Bp + i), cc = __ldg(Cp + i);
+            const float4 zero4 = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            const float4 bb = bc_ok ? __ldg(Bp + i) : zero4, cc = bc_ok ? __ldg(Cp + i) : zero4;
             B2[2 * i] = pack2(bb.x, bb.y); B2[2 * i + 1] = pack2(bb.z, bb.w);
             C2[2 * i] = pack2(cc.x, cc.y); C2[2 * i + 1] = pack2(cc.z, cc.w);
         }
@@ -155,12 +163,15 @@ __global__ void __launch_bounds__(kThreads, SSDQ_STREAM_MINB) ssd_update_stream_
         }
         const float dtv = dt_next, Dl = D_next;
         const float a = exp_spec(__fmul_rn(dtv, A_next));
-        if (item + 1 < last) {
+        if (item + 1 < last && SSDQ_RANGE_OK(p, DBG_ITEMS, item + 1, 1, items)) {
             const uint32_t h_n = (h + 1u == p.H) ? 0u : h + 1u;
             dt_next = __ldg(p.dt + item + 1);
             A_next = __ldg(p.A + h_n);
             D_next = (p.D && lis == 0) ? __ldg(p.D + h_n) : 0.0f;
         }
+        const uint64_t crow = (uint64_t)(c_y - p.y) - lis / (LPR / 4);
+        const bool mem_ok = SSDQ_RANGE_OK(p, DBG_STATE, crow * LPR + lis, (RPS - 1) * LPR + 1, state_vecs) && SSDQ_RANGE_OK(p, DBG_ROWS, crow, RPS, rows) &&
+                            SSDQ_RANGE_OK(p, DBG_SCALES, crow * SPR + (ROW_SCALE ? 0u : lis), (RPS - 1) * SPR + 1, scales);
         uint32_t acc_row = 0;
         uint64_t grp_row = 0;
         if constexpr (RULE == RULE_WEYL) acc_row = thr.weyl_acc0(grow_first);
@@ -210,8 +221,8 @@ __global__ void __launch_bounds__(kThreads, SSDQ_STREAM_MINB) ssd_update_stream_
             float v[EPL];
 #pragma unroll
             for (int i = 0; i < EPL / 2; ++i) unpack2(mul2_rn(hv[i], rinv2), v[2 * i], v[2 * i + 1]);
-            if constexpr (ROW_SCALE) { if (lis == 0) c_sc[k] = s; }
-            else c_sc[k * SPR] = s;
+            if constexpr (ROW_SCALE) { if (lis == 0 && mem_ok) c_sc[k] = s; }
+            else if (mem_ok) c_sc[k * SPR] = s;
 
             uint32_t acc[EPL];
             if constexpr (RULE == RULE_WEYL) {
@@ -230,7 +241,7 @@ __global__ void __launch_bounds__(kThreads, SSDQ_STREAM_MINB) ssd_update_stream_
                 }
                 grp_row += N / 4;
             }
-            c_codes[k * LPR] = round_pack16<FMT, RULE>(v, acc, top);
+            if (mem_ok) c_codes[k * LPR] = round_pack16<FMT, RULE>(v, acc, top);
             return __fadd_rn(d0, d1);
         };
 #pragma unroll
@@ -243,7 +254,7 @@ __global__ void __launch_bounds__(kThreads, SSDQ_STREAM_MINB) ssd_update_stream_
             const float d2 = process_row(g4 * 4 + 2, x4.z, s4.z);
             const float d3 = process_row(g4 * 4 + 3, x4.w, s4.w);
             const float tot = reduce4_over_slot<LPR>(d0, d1, d2, d3, lis);
-            if (y_writer) c_y[g4 * 4] = tot;
+            if (y_writer && mem_ok) c_y[g4 * 4] = tot;
         }
         c_codes += ROWS * LPR;
         c_sc += ROWS * SPR;

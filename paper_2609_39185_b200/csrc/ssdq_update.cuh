@@ -198,6 +198,8 @@ __global__ void __launch_bounds__(kThreads) ssd_update_kernel(const UpdateParams
     float Bv[EPL], Cv[EPL];
     {
         const size_t grp = (size_t)b * p.ngroups + h / p.heads_per_group;
+        (void)SSDQ_RANGE_OK(p, DBG_BC, grp * N + n0, EPL, bc_floats);
+        (void)SSDQ_RANGE_OK(p, DBG_ITEMS, item, 1, items);
         const float4* Bp = reinterpret_cast<const float4*>(p.Bm + grp * N + n0);
         const float4* Cp = reinterpret_cast<const float4*>(p.Cm + grp * N + n0);
 #pragma unroll
@@ -247,6 +249,11 @@ __global__ void __launch_bounds__(kThreads) ssd_update_kernel(const UpdateParams
         for (int u = 0; u < UNR; ++u) {
             const uint32_t k = k0 + u;
             ok[u] = item_ok && (k < p.rps) && (p_first + k < p.P);
+            if (ok[u]) {        // debug builds: the row's vector, x / y element and scale must lie inside the caller's buffers
+                ok[u] = SSDQ_RANGE_OK(p, DBG_STATE, (row_first + k) * LPR + lis, 1, state_vecs) && SSDQ_RANGE_OK(p, DBG_ROWS, row_first + k, 1, rows);
+                if constexpr (Fmt<FMT>::kScaled)
+                    ok[u] = ok[u] && SSDQ_RANGE_OK(p, DBG_SCALES, row_scale ? row_first + k : (row_first + k) * (N / 16) + lis, 1, scales);
+            }
             raw[u] = make_uint4(0u, 0u, 0u, 0u);
             xv[u] = 0.0f;
             sc[u] = 0.0f;
@@ -405,16 +412,25 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
     // cp.async.wait_group is all the synchronisation needed.
     __shared__ uint4 tile[RPS][kThreads];
     uint4* sp = reinterpret_cast<uint4*>(p.state) + row_first * LPR + lis;
+    // debug builds: everything this lane will touch, checked once (a lane that fails keeps running but accesses nothing)
+    bool mem_ok = SSDQ_RANGE_OK(p, DBG_STATE, row_first * LPR + lis, (RPS - 1) * LPR + 1, state_vecs) &&
+                  SSDQ_RANGE_OK(p, DBG_ROWS, row_first, RPS, rows) && SSDQ_RANGE_OK(p, DBG_ITEMS, item, 1, items) &&
+                  SSDQ_RANGE_OK(p, DBG_BC, (size_t)b * ((EXTRAS && p.ngroups > 1) ? p.ngroups : 1u) * N + n0, EPL, bc_floats);
+    if constexpr (Fmt<FMT>::kScaled)
+        mem_ok = mem_ok && SSDQ_RANGE_OK(p, DBG_SCALES, row_scale ? row_first : row_first * (N / 16) + lis, row_scale ? RPS : (RPS - 1) * (N / 16) + 1, scales);
 #pragma unroll
     for (int k = 0; k < RPS; ++k) {
         const uint32_t dst = (uint32_t)__cvta_generic_to_shared(&tile[k][threadIdx.x]);
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n cp.async.commit_group;" ::"r"(dst), "l"(sp + k * LPR) : "memory");
+        if (mem_ok) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n cp.async.commit_group;" ::"r"(dst), "l"(sp + k * LPR) : "memory");
     }
     float xv[RPS];
     float sc[Fmt<FMT>::kScaled ? RPS : 1];
 #pragma unroll
     for (int k = 0; k < RPS / GRP; ++k) {
-        if constexpr (GRP == 4) {
+        if (!mem_ok) {
+            xv[GRP * k] = 0.0f; xv[GRP * k + 1] = 0.0f;
+            if constexpr (GRP == 4) { xv[4 * k + 2] = 0.0f; xv[4 * k + 3] = 0.0f; }
+        } else if constexpr (GRP == 4) {
             const float4 x4 = __ldg(reinterpret_cast<const float4*>(p.x + row_first) + k);
             xv[4 * k] = x4.x; xv[4 * k + 1] = x4.y; xv[4 * k + 2] = x4.z; xv[4 * k + 3] = x4.w;
         } else {
@@ -424,7 +440,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
     }
     if constexpr (Fmt<FMT>::kScaled) {
 #pragma unroll
-        for (int k = 0; k < RPS; ++k) sc[k] = row_scale ? p.scales[row_first + k] : p.scales[(row_first + k) * (N / 16) + lis];
+        for (int k = 0; k < RPS; ++k) sc[k] = !mem_ok ? 0.0f : row_scale ? p.scales[row_first + k] : p.scales[(row_first + k) * (N / 16) + lis];
     }
     f32x2 B2[EPL / 2], C2[EPL / 2];
     {
@@ -433,12 +449,13 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
         const float4* Cp = reinterpret_cast<const float4*>(p.Cm + grp * N + n0);
 #pragma unroll
         for (int i = 0; i < EPL / 4; ++i) {
-            const float4 bb = __ldg(Bp + i), cc = __ldg(Cp + i);
+            const float4 zero4 = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            const float4 bb = mem_ok ? __ldg(Bp + i) : zero4, cc = mem_ok ? __ldg(Cp + i) : zero4;
             B2[2 * i] = pack2(bb.x, bb.y); B2[2 * i + 1] = pack2(bb.z, bb.w);
             C2[2 * i] = pack2(cc.x, cc.y); C2[2 * i + 1] = pack2(cc.z, cc.w);
         }
     }
-    float dtv = __ldg(p.dt + item);
+    float dtv = mem_ok ? __ldg(p.dt + item) : 0.0f;
     if constexpr (EXTRAS) {
         if (p.dt_bias) dtv = __fadd_rn(dtv, __ldg(p.dt_bias + h));
         if (p.dt_softplus) dtv = softplus_spec(dtv);
@@ -448,7 +465,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
     float gate[RPS / GRP];
 #pragma unroll
     for (int g4 = 0; g4 < RPS / GRP; ++g4)
-        gate[g4] = (EXTRAS && p.z && y_writer) ? __ldg(p.z + row_first + g4 * GRP + lis / (LPR / GRP)) : 0.0f;
+        gate[g4] = (EXTRAS && p.z && y_writer && mem_ok) ? __ldg(p.z + row_first + g4 * GRP + lis / (LPR / GRP)) : 0.0f;
     const float a = exp_spec(__fmul_rn(dtv, __ldg(p.A + h)));
     const f32x2 a2 = pack2(a, a);
     const float Dl = (p.D && lis == 0) ? __ldg(p.D + h) : 0.0f;     // the skip term enters the dot on one lane
@@ -503,20 +520,20 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
                 const f32x2 rinv2 = pack2(rinv, rinv);
 #pragma unroll
                 for (int i = 0; i < EPL / 2; ++i) unpack2(mul2_rn(hn2[i], rinv2), hv[2 * i], hv[2 * i + 1]);
-                if (row_scale) { if (lis == 0) p.scales[row_first + k] = s; }
-                else p.scales[(row_first + k) * (N / 16) + lis] = s;
+                if (row_scale) { if (lis == 0 && mem_ok) p.scales[row_first + k] = s; }
+                else if (mem_ok) p.scales[(row_first + k) * (N / 16) + lis] = s;
             }
             if constexpr (RULE == RULE_SR_HASH) acc_row = thr.hash_key0(grow_first + k, hash_base, key1);
             const uint4 packed = round_pack_lane<FMT, RULE>(hv, acc_row, p.weyl.mul_col, (uint32_t)grp_row,
                                                              (uint32_t)(grp_row >> 32), step_t, p.layer, key0, key1, p.scale_top);
-            sp[k * LPR] = packed;
+            if (mem_ok) sp[k * LPR] = packed;
             if constexpr (RULE == RULE_WEYL) acc_row += thr.row_mul;
             if constexpr (RULE == RULE_SR) grp_row += N / 4;
         }
         float tot;
         if constexpr (GRP == 4) tot = reduce4_over_slot<LPR>(dots[0], dots[1], dots[2], dots[3], lis);
         else tot = reduce2_over_slot<LPR>(dots[0], dots[1], lis);
-        if (y_writer) p.y[row_first + g4 * GRP + lis / (LPR / GRP)] = (EXTRAS && p.z) ? __fmul_rn(tot, silu(gate[g4])) : tot;
+        if (y_writer && mem_ok) p.y[row_first + g4 * GRP + lis / (LPR / GRP)] = (EXTRAS && p.z) ? __fmul_rn(tot, silu(gate[g4])) : tot;
     }
 }
 

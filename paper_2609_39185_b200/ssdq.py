@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libssdq.so")
 EXPORTS = ("weyl_offsets_init", "ssdq_thresholds_materialize", "ssd_state_update", "quantize_store",
            "ssdq_dequantize", "ssd_decode_run", "ssd_decode_run_host", "ssd_replay_step", "ssd_decode_run_checkpointed",
            "ssd_decode_graph_create", "ssd_decode_graph_launch", "ssd_decode_graph_destroy", "ssdq_state_error_workspace_bytes", "ssdq_state_error",
-           "ssdq_state_error_static", "ssdq_readout_kl", "ssdq_copy", "ssdq_last_kernel", "ssdq_last_error", "ssdq_launch_count")
+           "ssdq_state_error_static", "ssdq_readout_kl", "ssdq_copy", "ssdq_debug_status", "ssdq_last_kernel", "ssdq_last_error", "ssdq_launch_count")
 
 _u32, _u64, _i32, _vp = ctypes.c_uint32, ctypes.c_uint64, ctypes.c_int32, ctypes.c_void_p
 
@@ -51,6 +51,8 @@ class StepInputs(ctypes.Structure):
                 ("z", _vp), ("stride_z", _u64)]
 
 
+DEBUG_LIB_PATH = os.path.join(_HERE, "libssdq_debug.so")
+
 _lib = None
 
 
@@ -58,10 +60,16 @@ def lib() -> ctypes.CDLL:
     """Load libssdq.so (built by ``python -m paper_2609_39185_b200.build``); raises if it is missing."""
     global _lib
     if _lib is None:
-        if not os.path.exists(LIB_PATH):
-            raise ImportError(f"{LIB_PATH} is missing: build the CUDA extension first "
+        _lib = _load(LIB_PATH)
+    return _lib
+
+
+def _load(path) -> ctypes.CDLL:
+    if True:
+        if not os.path.exists(path):
+            raise ImportError(f"{path} is missing: build the CUDA extension first "
                               "(python -m paper_2609_39185_b200.build); there is no CPU fallback")
-        L = ctypes.CDLL(LIB_PATH)
+        L = ctypes.CDLL(path)
         L.weyl_offsets_init.restype = ctypes.c_int
         L.weyl_offsets_init.argtypes = [ctypes.POINTER(Weyl), _u32, _u32, _u32]
         L.ssdq_thresholds_materialize.restype = ctypes.c_int
@@ -106,8 +114,32 @@ def lib() -> ctypes.CDLL:
         L.ssdq_last_error.argtypes = []
         L.ssdq_launch_count.restype = _u64
         L.ssdq_launch_count.argtypes = []
-        _lib = L
-    return _lib
+        L.ssdq_debug_status.restype = ctypes.c_int
+        L.ssdq_debug_status.argtypes = [ctypes.POINTER(_u32 * 4), ctypes.c_int]
+    return L
+
+
+class debug_library:
+    """Context manager: inside it every call of this module goes to the bounds-checking build of the library
+    (libssdq_debug.so, from ``python -m paper_2609_39185_b200.build --debug``); debug_status() reads its status words."""
+
+    def __enter__(self):
+        global _lib
+        self._saved = _lib
+        _lib = _load(DEBUG_LIB_PATH)
+        return self
+
+    def __exit__(self, *exc):
+        global _lib
+        _lib = self._saved
+        return False
+
+
+def debug_status(reset: bool = True):
+    """(code, index, block) of the first out-of-range access the bounds-checking build saw, or (0, 0, 0)."""
+    out = (_u32 * 4)()
+    _check(lib().ssdq_debug_status(ctypes.byref(out), int(reset)))
+    return int(out[0]), int(out[1]) | (int(out[2]) << 32), int(out[3])
 
 
 def _check(status):

@@ -139,3 +139,17 @@ def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(ssdq, "LIB_PATH", "/nonexistent/libssdq.so")
     with pytest.raises(ImportError):
         ssdq.lib()
+
+
+def test_debug_status_is_refused_by_the_release_build(lib):
+    out = (ctypes.c_uint32 * 4)()
+    assert lib.ssdq_debug_status(ctypes.byref(out), 1) == ssdq.ERR_UNSUPPORTED
+    assert b"SSDQ_DEBUG" in lib.ssdq_last_error()
+
+
+def test_the_bounds_checking_build_exports_the_same_symbols():
+    path = ssdq_build.build(debug=True)
+    assert path.endswith("libssdq_debug.so")
+    dbg = ctypes.CDLL(path)
+    for n in ssdq.EXPORTS:
+        assert hasattr(dbg, n), n
