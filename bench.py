@@ -34,8 +34,12 @@ FALLBACK_HBM_GBS = 6650.0      # an earlier stream-copy measurement on this machine
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the fused update kernel from the one-kernel ncu
 # captures summarised under profiles/ (same kernel and per-layer shape as the benchmark's launches; see NCU_TRAFFIC_SOURCE).
 # A launch ends with part of its last writes still in L2, so the write term undercounts by up to the L2 size.
-NCU_TRAFFIC_BYTES = {}
-NCU_TRAFFIC_SOURCE = "profiles/ssd_update_tile_kernel_bf16_config5.md (one launch, 2 layers resident)"
+NCU_TRAFFIC_BYTES = {(5, "weyl"): 272_967_936 + 215_749_376, (5, "rtn"): 272_995_072 + 215_929_088,
+                     (3, "weyl"): 85_321_216 + 26_518_272, (3, "rtn"): 85_298_176 + 28_177_408,
+                     (4, "weyl"): 17_901_056 + 0, (4, "rtn"): 17_884_672 + 0}
+NCU_TRAFFIC_SOURCE = {5: "profiles/ssd_update_tile_kernel_bf16_config5.md (one launch, 2 layers resident; ~57 MB of the writes still in L2 at launch end)",
+                      3: "profiles/ssd_update_tile_kernel_fp16_config3.md (state smaller than L2: writes mostly stay there)",
+                      4: "profiles/ssd_update_stream_kernel_e4m3_int8.md (state L2-resident: no DRAM writes within a launch)"}
 
 
 def measured_peak(path=None):
@@ -382,7 +386,7 @@ def main():
             "pct_of_measured_copy": 100.0 * gbs / world / peak,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": None if (args.batch or args.format) else NCU_TRAFFIC_BYTES.get((cfg.index, args.rule)),
-                         "traffic_source": NCU_TRAFFIC_SOURCE, "kernel": ssdq.last_kernel(), "peak_source": peak_src,
+                         "traffic_source": NCU_TRAFFIC_SOURCE.get(cfg.index), "kernel": ssdq.last_kernel(), "peak_source": peak_src,
                          "algorithmic_bytes_per_launch": bytes_per_launch, "launch_us": launch_secs * 1e6},
             "clocks": clocks, "gpu_launches": int(launches)}
 

@@ -102,8 +102,8 @@ typedef struct {
     uint64_t sr_seed;    /* Philox key when rule == SSDQ_SR_PHILOX */
     uint32_t layer;      /* layer index in the SR counter (the Weyl layer term sits in weyl.base) */
     uint32_t batch_index_base;  /* global index of local sequence 0 */
-    /* The rest of a production selective-state-update signature (Appendix B "Runners": grouped B and C, gating as
-     * in the reference implementations).  All optional: zero / NULL gives the plain step. */
+    /* The rest of a production selective-state-update signature (Appendix B "Runners" keeps the grouped B and C and
+     * the output gate of the Mamba implementations it follows).  All optional: zero / NULL gives the plain step. */
     const float* dt_bias;/* [H] or NULL: added to dt (one rounded add) */
     const float* z;      /* [B, H, P] or NULL: y <- y * z * sigmoid(z) */
     uint32_t dt_softplus;/* 1: dt <- softplus_spec(dt + dt_bias), the library's fixed binary32 softplus */

@@ -72,8 +72,8 @@ int int_qmax(int fmt) {
 bool has_block_scale(int fmt) { return fmt == FMT_E4M3 || is_int_format(fmt); }
 
 // ------------------------------------------------------------------------------------------
-// Thresholds.  U is a 24-bit integer, u = U / 2^24 (Appendix B "Dithers": "the top 24 bits
-// divided by 2^24").
+// Thresholds.  U is a 24-bit integer, the leading 24 bits of the 32-bit accumulator, and u = U / 2^24
+// (Appendix B "Dithers").
 // ------------------------------------------------------------------------------------------
 
 // Appendix B "Dithers", hardware form.  The four multipliers are the decimal constants printed
@@ -109,7 +109,7 @@ void philox4x32_10(const uint32_t ctr_in[4], const uint32_t key_in[2], uint32_t 
 }
 
 // Integer-hash SR (Section 6.5 "Cost": SR driven by a cheap integer hash is as accurate as Philox SR; Appendix B
-// "Decode regime": u = fmix32(i * 0x9E3779B1 + t * 0x85EBCA77 + ...) / 2^32 truncated to 24 bits).  fmix32 is the
+// "Decode regime": the hash fmix32(i * 0x9E3779B1 + t * 0x85EBCA77 + ...), of which 24 bits are kept).  fmix32 is the
 // 32-bit finaliser of MurmurHash3.  The paper elides the remaining terms; this build continues the same family
 // of odd multipliers for layer and seed and folds in the high half of a 64-bit entry index.
 uint32_t fmix32(uint32_t h) {
@@ -354,8 +354,8 @@ void oracle_exp_spec_array(const float* z, uint64_t n, float* out) {
 // state  : [B, H, P, N] codes of `fmt` (FMT_FP32: floats, no rounding = the fp32-state twin)
 // scales : E4M3 only, [B, H, P, N / scale_block] floats, or [B, H] when scale_block == P * N
 // x [B,H,P], dt [B,H], A [H] or [H,N] (a_per_state), Bm, Cm [B,G,N], D [H] or null, y [B,H,P]
-// The rest of a production selective-state-update signature (Appendix B "Runners": grouped B and C, gating as in
-// the reference implementations): dt_bias [H] or null, dt_softplus (dt <- softplus_spec(dt + dt_bias)), ngroups G
+// The rest of a production selective-state-update signature (Appendix B "Runners" keeps the grouped B and C and the
+// output gate of the Mamba implementations it follows): dt_bias [H] or null, dt_softplus (dt <- softplus_spec(dt + dt_bias)), ngroups G
 // (head h reads group h / (H / G)), z [B,H,P] or null (y <- y * z * sigmoid(z)).
 // Returns 0, or -1 on an argument the oracle does not define.
 int oracle_state_update(void* state, float* scales, int fmt, uint32_t scale_block,

@@ -3,8 +3,8 @@ code for code.
 
 The dithered BF16 and FP16 stores run on the hardware stochastic-rounding converts and the E4M3 dither on an
 integer form plus a truncating convert, so the rounding of each format is checked on all of its inputs rather than on
-samples (Section 2, "Rounding with a threshold": the rule applied on the local grid of representable values;
-Appendix B "Formats").  Thresholds: one value for all entries (0, 2^24 - 1, one mid-range value: a Weyl descriptor whose row and
+samples (Section 2, "Rounding with a threshold": floating-point formats round on the grid spacing of the value's own
+binade; Appendix B "Formats").  Thresholds: one value for all entries (0, 2^24 - 1, one mid-range value: a Weyl descriptor whose row and
 column multipliers are zero gives every entry the accumulator `base`) and the real Weyl streams at a large write index.
 
 BF16, FP16: all 2^32 - 2^24 finite patterns.  E4M3, INT8: all patterns with |v| <= 448 (127), each block of 16 entries

@@ -31,7 +31,7 @@ def test_weyl_sequence_starts_618_236_854():
 
 def test_weyl_integer_form_tracks_float_form():
     # Appendix B "Dithers": u = frac(o_{r,c} + t*alpha) with the decimal generators; the 32-bit
-    # accumulator uses those constants times 2^32, so each term is off by at most half a unit of 2^-32.
+    # accumulator holds each generator scaled by 2^32 and rounded, so each term is off by at most half a unit of 2^-32.
     rng = np.random.default_rng(0)
     for _ in range(2000):
         r, c = int(rng.integers(0, 1 << 20)), int(rng.integers(0, 128))
