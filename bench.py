@@ -237,9 +237,10 @@ def formats_table(cfg, peak, xs, dts, Bs, Cs, layers=2, rounds=7, reps=20):
     out = {"note": f"per-layer shape of config {cfg.index}, {layers} layers resident, {rounds} interleaved rounds of {reps} steps, median"}
     ring = tuple(t[:, :layers].contiguous() for t in (xs, dts, Bs, Cs))
     sin = ssdq.make_step_inputs(*ring, torch.empty_like(ring[0]))
-    for name in ("bf16", "fp16", "e4m3", "int8"):
-        fmt = {v: k for k, v in workloads.FORMAT_NAMES.items()}[name]
-        c = replace(cfg, n_layers=layers, fmt=fmt, scale_block=cfg.weyl_block if fmt in workloads.SCALED_FORMATS else 0)
+    for name in ("bf16", "fp16", "e4m3", "int8", "int8_block16"):      # scaled stores: one scale per row of N; _block16: per 16 entries
+        fmt = {v: k for k, v in workloads.FORMAT_NAMES.items()}[name.split("_")[0]]
+        sb = 0 if fmt not in workloads.SCALED_FORMATS else 16 if name.endswith("_block16") else cfg.weyl_block
+        c = replace(cfg, n_layers=layers, fmt=fmt, scale_block=sb)
         stack = Stack(c, RULE_IDS["rtn"])
         stack.run(1, 5, sin)
         torch.cuda.synchronize()
