@@ -541,6 +541,15 @@ ssdq_status ssd_decode_graph_create(ssdq_graph** out, const ssdq_update_desc* la
                                            in->Cm + k * in->stride_C, in->y + k * in->stride_y, in->z ? in->z + k * in->stride_z : nullptr);
             if (rc != SSDQ_OK) return rc;
         }
+    // one-time set-up of the kernels the layers will use (function attributes, occupancy queries) happens here, before the
+    // capture: nothing but launches is issued while the stream is capturing
+    for (uint32_t l = 0; l < n_layers; ++l) {
+        ssdq::UpdateParams p = make_params(&layers[l], 1u);
+        p.x = in->x; p.y = in->y; p.z = in->z;
+        p.prepare_only = 1;
+        const cudaError_t pe = launch_update(p, layers[l].format, layers[l].rule, layers[l].a_per_state != 0, nullptr);
+        if (pe != cudaSuccess) return fail(SSDQ_ERR_CUDA, "state-update kernel set-up: %s", cudaGetErrorString(pe));
+    }
     cudaStream_t cs = nullptr;
     cudaError_t e = cudaStreamCreateWithFlags(&cs, cudaStreamNonBlocking);
     if (e != cudaSuccess) return fail(SSDQ_ERR_CUDA, "cudaStreamCreate: %s", cudaGetErrorString(e));

@@ -157,6 +157,7 @@ cudaError_t try_launch_headscale(const UpdateParams& p, cudaStream_t stream, boo
         if (p.P == nslot * (R)) {                                                                  \
             launched = true;                                                                       \
             note_kernel(3);                                                                        \
+            if (p.prepare_only) return cudaSuccess;                                                \
             ssd_update_headscale_kernel<FMT, RULE, LPR, R><<<grid, kThreads, 0, stream>>>(p);      \
             return cudaGetLastError();                                                             \
         }

@@ -50,6 +50,7 @@ struct UpdateParams {
     uint32_t rps;            // rows per slot
     WeylConst weyl;
     uint64_t sr_seed;
+    uint32_t prepare_only;   // host side only: pick the kernel and do its one-time set-up (attributes, occupancy), launch nothing
 #ifdef SSDQ_DEBUG
     DebugBounds dbg;
 #endif

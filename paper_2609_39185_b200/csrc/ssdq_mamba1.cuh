@@ -166,6 +166,7 @@ cudaError_t try_launch_mamba1(const UpdateParams& p, cudaStream_t stream, bool& 
         chunks = (p.B + q.rps - 1) / q.rps;
         launched = true;
         note_kernel(4);
+        if (p.prepare_only) return cudaSuccess;
         ssd_update_mamba1_kernel<FMT, RULE><<<dim3(tiles, chunks), kThreads, 0, stream>>>(q);
         return cudaGetLastError();
     }

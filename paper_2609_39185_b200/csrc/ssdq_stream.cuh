@@ -303,6 +303,7 @@ inline cudaError_t launch_stream(const UpdateParams& p, cudaStream_t stream) {
     uint32_t grid = (uint32_t)(ctas * sms);            // one wave of resident CTAs
     if (grid > p.n_items) grid = p.n_items;
     note_kernel(2);
+    if (p.prepare_only) return cudaSuccess;
     ssd_update_stream_kernel<FMT, RULE, LPR, RPS, STAGES, ROW_SCALE><<<grid, kThreads, stream_smem_bytes<RPS, STAGES>(), stream>>>(p);
     return cudaGetLastError();
 }

@@ -582,6 +582,7 @@ inline cudaError_t launch_update_one(const UpdateParams& p, cudaStream_t stream)
 #define SSDQ_TILE_CASE(R)                                                                                          \
             if (q.P == nslot * (R)) {                                                                              \
                 note_kernel(1);                                                                                    \
+                if (q.prepare_only) return cudaSuccess;                                                            \
                 if (extras) ssd_update_tile_kernel<FMT, RULE, LPR, R, true><<<tile_grid, kThreads, 0, stream>>>(q);  \
                 else ssd_update_tile_kernel<FMT, RULE, LPR, R, false><<<tile_grid, kThreads, 0, stream>>>(q);       \
                 return cudaGetLastError();                                                                         \
@@ -600,6 +601,7 @@ inline cudaError_t launch_update_one(const UpdateParams& p, cudaStream_t stream)
     q.rps = (q.P + spi - 1) / spi;
     const uint32_t grid = (q.n_items + q.items_per_cta - 1) / q.items_per_cta;
     note_kernel(0);
+    if (q.prepare_only) return cudaSuccess;
     ssd_update_kernel<FMT, RULE, LPR, APS><<<grid, kThreads, 0, stream>>>(q);
     return cudaGetLastError();
 }

@@ -508,3 +508,41 @@ def test_graph_replay_equals_the_plain_driver(rule):
         assert torch.equal(s1[l], s2[l])
     assert torch.equal(y1, y2)
     graph.close()
+
+
+def test_graph_replay_on_the_persistent_kernel():
+    """The replayable graph over the one-byte persistent kernel (whose one-time set-up must happen before the capture
+    begins: this instantiation -- E4M3, hash SR, heads of 128 rows, one scale per 16 entries -- is launched nowhere else
+    before): equal to the plain driver."""
+    from dataclasses import replace
+    cfg = replace(workloads.CONFIGS[4], batch=2, nheads=6, headdim=128, scale_block=16)
+    L, ring, spl, reps = 2, 2, 2, 3
+    rule = ssdq.SR_HASH
+    params = [workloads.layer_params(cfg, l, l) for l in range(L)]
+    ins = [[workloads.step_inputs(cfg, t + 1, l, l) for l in range(L)] for t in range(ring)]
+    stack = lambda i: to_dev(np.stack([np.stack([ins[t][l][i] for l in range(L)]) for t in range(ring)]))
+    xs, dts, Bs, Cs = (stack(i) for i in range(4))
+
+    def fresh():
+        states = [torch.zeros(cfg.state_shape, dtype=torch.uint8, device="cuda") for _ in range(L)]
+        scales = [torch.full((cfg.entries_per_layer // 16,), float(np.finfo(np.float32).tiny), device="cuda") for _ in range(L)]
+        descs = [ssdq.make_desc(states[l], scales[l], cfg.fmt, A=to_dev(params[l][0]), D=to_dev(params[l][1]), rule=rule,
+                                weyl=ssdq.weyl_offsets_init(l, 0, cfg.weyl_block), sr_seed=l, layer=l, scale_block=16) for l in range(L)]
+        return states, scales, descs
+
+    s2, c2, d2 = fresh()
+    y2 = torch.zeros_like(xs)
+    counter = torch.zeros(1, dtype=torch.int32, device="cuda")
+    graph = ssdq.DecodeGraph(d2, spl, ssdq.make_step_inputs(xs, dts, Bs, Cs, y2), counter)     # first use of the instantiation
+    for _ in range(reps):
+        graph.launch()
+    torch.cuda.synchronize()
+    assert ssdq.last_kernel() == "ssd_update_stream_kernel"
+    s1, c1, d1 = fresh()
+    y1 = torch.zeros_like(xs)
+    ssdq.ssd_decode_run(d1, 1, spl * reps, ssdq.make_step_inputs(xs, dts, Bs, Cs, y1))
+    torch.cuda.synchronize()
+    for l in range(L):
+        assert torch.equal(s1[l], s2[l]) and torch.equal(c1[l], c2[l])
+    assert torch.equal(y1, y2)
+    graph.close()
