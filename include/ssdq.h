@@ -18,8 +18,9 @@
  *   - Every argument check happens before any launch; a failed check launches nothing.
  *   - Return value: SSDQ_OK or a negative ssdq_status; ssdq_last_error() gives a thread-local text.
  *   - Indices that feed the thresholds are GLOBAL: entry (b, h, p, n) of a layer has flat index
- *     ((( b + batch_index_base) * H + h) * P + p) * N + n, so a batch shard reproduces the bits of
- *     the unsharded run.
+ *     ((( b + batch_index_base) * H_global + h + head_index_base) * P + p) * N + n, with H_global =
+ *     nheads_global (or H when that field is 0), so a shard of the batch, of the heads, or of both
+ *     reproduces the bits of the unsharded run.  All tensors of a call hold the shard only.
  *   - All inputs must be finite.  Binary32 subnormals are honoured (no flush to zero).
  */
 #ifndef SSDQ_H_
@@ -107,7 +108,12 @@ typedef struct {
     const float* dt_bias;/* [H] or NULL: added to dt (one rounded add) */
     const float* z;      /* [B, H, P] or NULL: y <- y * z * sigmoid(z) */
     uint32_t dt_softplus;/* 1: dt <- softplus_spec(dt + dt_bias), the library's fixed binary32 softplus */
-    uint32_t ngroups;    /* G > 1: Bm, Cm are [B, G, N] and head h reads group h / (H / G); 0 or 1: one group */
+    uint32_t ngroups;    /* G > 1: Bm, Cm are [B, G, N] and head h reads group h / (H / G); 0 or 1: one group.
+                            Heads and groups are those of this call's tensors (a head shard carries its own groups). */
+    /* Head shard (tensor parallel): this call holds heads head_index_base .. head_index_base + H - 1 of a layer with
+     * nheads_global heads.  Only the threshold indices change.  0, 0 = the call holds every head. */
+    uint32_t head_index_base;   /* global index of local head 0 */
+    uint32_t nheads_global;     /* 0 = nheads; otherwise >= head_index_base + nheads */
 } ssdq_update_desc;
 
 /* One fused decode step of one layer (Eq. 1, readout, Eq. 2), in place, one kernel launch:

@@ -72,7 +72,7 @@ def lib() -> ctypes.CDLL:
         L.oracle_exp_spec_array.argtypes = [vp, u64, vp]
         L.oracle_state_update.restype = i32
         L.oracle_state_update.argtypes = [vp, vp, i32, u32, u32, u32, u32, u32, vp, vp, vp, i32, vp, vp, vp, vp,
-                                          i32, u32, u32, u32, u64, u32, u32, vp, i32, u32, vp]
+                                          i32, u32, u32, u32, u64, u32, u32, vp, i32, u32, vp, u32, u32]
         L.oracle_softplus_spec.restype = f32
         L.oracle_softplus_spec.argtypes = [f32]
         L.oracle_quantize_store.restype = i32
@@ -178,12 +178,14 @@ def softplus_spec(x):
 
 def state_update(state, scales, fmt, scale_block, x, dt, A, Bm, Cm, D, rule, step_t, *, layer=0,
                  weyl_seed=0, weyl_block=16, sr_seed=0, batch_index_base=0, dt_bias=None, dt_softplus=False,
-                 ngroups=1, z=None):
+                 ngroups=1, z=None, head_index_base=0, nheads_global=0):
     """One decode step of one layer, in place on `state` (and `scales`).  Returns y [B,H,P] float32.
 
     state [B,H,P,N] of CODE_DTYPE[fmt] (float32 viewed as uint32 for FP32); x [B,H,P]; dt [B,H];
     A [H] or [H,N]; Bm, Cm [B,N] (or [B,G,N] with ngroups=G); D [H] or None; dt_bias [H] or None; with
     dt_softplus the step size is softplus_spec(dt + dt_bias); z [B,H,P] or None gates y by z * sigmoid(z).
+    The arrays may hold a slice of the layer: sequences from batch_index_base on, heads from head_index_base on out of
+    nheads_global (0 = H); the thresholds are drawn at the entry's index in the whole layer.
     """
     Bsz, H, P, N = state.shape
     assert state.flags.c_contiguous and state.dtype == CODE_DTYPE[fmt]
@@ -201,7 +203,7 @@ def state_update(state, scales, fmt, scale_block, x, dt, A, Bm, Cm, D, rule, ste
     rc = lib().oracle_state_update(_ptr(state), _ptr(scales), fmt, scale_block, Bsz, H, P, N, _ptr(x), _ptr(dt),
                                    _ptr(A), a_per_state, _ptr(Bm), _ptr(Cm), _ptr(D), _ptr(y), rule, layer,
                                    weyl_seed, weyl_block, sr_seed, batch_index_base, step_t, _ptr(dt_bias),
-                                   int(bool(dt_softplus)), ngroups, _ptr(z))
+                                   int(bool(dt_softplus)), ngroups, _ptr(z), head_index_base, nheads_global)
     if rc != 0:
         raise ValueError("oracle_state_update: undefined argument combination")
     return y

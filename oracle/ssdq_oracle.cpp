@@ -357,6 +357,8 @@ void oracle_exp_spec_array(const float* z, uint64_t n, float* out) {
 // The rest of a production selective-state-update signature (Appendix B "Runners" keeps the grouped B and C and the
 // output gate of the Mamba implementations it follows): dt_bias [H] or null, dt_softplus (dt <- softplus_spec(dt + dt_bias)), ngroups G
 // (head h reads group h / (H / G)), z [B,H,P] or null (y <- y * z * sigmoid(z)).
+// head_index_base, nheads_global: the call holds heads head_index_base .. head_index_base + H - 1 of a layer with
+// nheads_global heads (0 = H); like batch_index_base they only enter the entry index that the thresholds are drawn from.
 // Returns 0, or -1 on an argument the oracle does not define.
 int oracle_state_update(void* state, float* scales, int fmt, uint32_t scale_block,
                         uint32_t B, uint32_t H, uint32_t P, uint32_t N,
@@ -364,8 +366,11 @@ int oracle_state_update(void* state, float* scales, int fmt, uint32_t scale_bloc
                         const float* Bm, const float* Cm, const float* D, float* y,
                         int rule, uint32_t layer, uint32_t weyl_seed, uint32_t weyl_block, uint64_t sr_seed,
                         uint32_t batch_index_base, uint32_t step_t,
-                        const float* dt_bias, int dt_softplus, uint32_t ngroups, const float* z) {
+                        const float* dt_bias, int dt_softplus, uint32_t ngroups, const float* z,
+                        uint32_t head_index_base, uint32_t nheads_global) {
     if (ngroups == 0) ngroups = 1;
+    if (nheads_global == 0) nheads_global = H;
+    if (head_index_base + H > nheads_global) return -1;
     if (H % ngroups != 0) return -1;
     const uint32_t heads_per_group = H / ngroups;
     if (has_block_scale(fmt)) {
@@ -425,7 +430,8 @@ int oracle_state_update(void* state, float* scales, int fmt, uint32_t scale_bloc
             }
             for (uint64_t i = s0; i < s0 + blk; ++i) {
                 const uint64_t local = (uint64_t)bh * head_elems + i;
-                const uint64_t flat = (uint64_t)batch_index_base * H * head_elems + local;
+                // the index of the entry in the whole layer, of which this call may hold a slice of the batch and of the heads
+                const uint64_t flat = (((uint64_t)batch_index_base + b) * nheads_global + head_index_base + h) * head_elems + i;
                 const float v = has_block_scale(fmt) ? hp[i] * rinv : hp[i];
                 const uint32_t U = threshold_u24(rp, flat, step_t);
                 store_code(state, local, fmt, encode(round_on_grid(v, fmt, rule, U), fmt));

@@ -70,6 +70,12 @@ ssdq_status check_layer(const ssdq_update_desc* d) {
     if (d->D && !aligned4(d->D)) return fail(SSDQ_ERR_ALIGN, "D is misaligned");
     if (d->dt_bias && !aligned4(d->dt_bias)) return fail(SSDQ_ERR_ALIGN, "dt_bias is misaligned");
     if (d->ngroups > 1 && d->nheads % d->ngroups != 0) return fail(SSDQ_ERR_SHAPE, "nheads must be a multiple of ngroups");
+    if (d->nheads_global == 0 ? d->head_index_base != 0
+                              : (d->nheads_global < d->nheads || d->head_index_base > d->nheads_global - d->nheads))
+        return fail(SSDQ_ERR_SHAPE, "head shard [%u, %u + %u) does not fit in nheads_global = %u", d->head_index_base, d->head_index_base,
+                    d->nheads, d->nheads_global);
+    if ((uint64_t)(d->nheads_global ? d->nheads_global - d->nheads : 0u) * d->headdim > 0xFFFFFFFFull)
+        return fail(SSDQ_ERR_SHAPE, "nheads_global * headdim is too large");
     if (format_scaled(d->format)) {
         if (!d->scales) return fail(SSDQ_ERR_NULL, "E4M3 and INTb stores need a scale array");
         if (!aligned4(d->scales)) return fail(SSDQ_ERR_ALIGN, "scales are misaligned");
@@ -128,7 +134,12 @@ ssdq::UpdateParams make_params(const ssdq_update_desc* d, uint32_t step_t) {
     p.scale_block = d->scale_block;
     p.scale_top = scale_top(d->format);
     p.inv_scale_top = 1.0f / p.scale_top;
-    p.step_t = step_t; p.layer = d->layer; p.batch_base = d->batch_index_base;
+    p.step_t = step_t; p.layer = d->layer;
+    {
+        const uint32_t Hg = d->nheads_global ? d->nheads_global : d->nheads;
+        p.row_off0 = ((uint64_t)d->batch_index_base * Hg + d->head_index_base) * d->headdim;
+        p.row_skip = (Hg - d->nheads) * d->headdim;
+    }
     p.weyl = weyl_const(d->weyl);
     p.sr_seed = d->sr_seed;
 #ifdef SSDQ_DEBUG
@@ -252,9 +263,11 @@ ssdq_status ssd_state_update(const ssdq_update_desc* d, uint32_t step_t, void* s
                        "state-update kernel");
 }
 
-ssdq_status quantize_store(const float* src, void* dst_codes, float* dst_scales, uint64_t n_rows, uint32_t row_len,
-                   uint32_t scale_block, int format, int rule, const ssdq_weyl* weyl, uint64_t sr_seed, uint32_t layer,
-                   uint64_t row_index_base, uint32_t step_t, void* stream) {
+// quantize_store with the row mapping of a head shard: global row = row_index_base + row + (row / rows_per_seq) * row_skip
+// (rows_per_seq == 0: rows are contiguous in the global view).
+static ssdq_status quantize_rows(const float* src, void* dst_codes, float* dst_scales, uint64_t n_rows, uint32_t row_len,
+                                 uint32_t scale_block, int format, int rule, const ssdq_weyl* weyl, uint64_t sr_seed, uint32_t layer,
+                                 uint64_t row_index_base, uint64_t rows_per_seq, uint32_t row_skip, uint32_t step_t, void* stream) {
     if (!format_known(format)) return fail(SSDQ_ERR_UNSUPPORTED, "unknown format %d", format);
     if (rule < SSDQ_RTN || rule > SSDQ_SR_HASH) return fail(SSDQ_ERR_UNSUPPORTED, "unknown rule %d", rule);
     if (!dstate_supported(format, row_len)) return fail(SSDQ_ERR_UNSUPPORTED, "row_len %u is not supported for format %d", row_len, format);
@@ -273,7 +286,15 @@ ssdq_status quantize_store(const float* src, void* dst_codes, float* dst_scales,
     }
     p.src = src; p.codes = dst_codes; p.scales = dst_scales; p.n_rows = n_rows; p.row_len = row_len;
     p.scale_block = scale_block; p.scale_top = scale_top(format); p.step_t = step_t; p.layer = layer; p.row_base = row_index_base; p.sr_seed = sr_seed;
+    p.rows_per_seq = row_skip ? rows_per_seq : 0; p.row_skip = row_skip;
     return cuda_result(ssdq::launch_quantize(p, kernel_format(format), rule, static_cast<cudaStream_t>(stream)), "quantize kernel");
+}
+
+ssdq_status quantize_store(const float* src, void* dst_codes, float* dst_scales, uint64_t n_rows, uint32_t row_len,
+                   uint32_t scale_block, int format, int rule, const ssdq_weyl* weyl, uint64_t sr_seed, uint32_t layer,
+                   uint64_t row_index_base, uint32_t step_t, void* stream) {
+    return quantize_rows(src, dst_codes, dst_scales, n_rows, row_len, scale_block, format, rule, weyl, sr_seed, layer, row_index_base,
+                         0, 0, step_t, stream);
 }
 
 ssdq_status ssd_replay_step(const float* w, const float* decay, uint32_t rows_per_decay, void* codes, float* scales, uint64_t n_rows,
@@ -346,8 +367,10 @@ ssdq_status ssd_decode_run_checkpointed(const ssdq_update_desc* layers, float* c
             if ((i + 1) % every != 0) continue;
             // every `every`-th write is rounded into the store (Eq. 2 under the layer's rule) and read back
             const uint64_t n_rows = (uint64_t)d.batch * d.nheads * d.headdim;
-            rc = quantize_store(work_fp32[l], d.state, d.scales, n_rows, d.dstate, d.scale_block, d.format, d.rule, &d.weyl,
-                                d.sr_seed, d.layer, (uint64_t)d.batch_index_base * d.nheads * d.headdim, t, stream);
+            const uint32_t Hg = d.nheads_global ? d.nheads_global : d.nheads;
+            rc = quantize_rows(work_fp32[l], d.state, d.scales, n_rows, d.dstate, d.scale_block, d.format, d.rule, &d.weyl,
+                               d.sr_seed, d.layer, ((uint64_t)d.batch_index_base * Hg + d.head_index_base) * d.headdim,
+                               (uint64_t)d.nheads * d.headdim, (Hg - d.nheads) * d.headdim, t, stream);
             if (rc != SSDQ_OK) return rc;
             rc = ssdq_dequantize(d.state, d.scales, n_rows * d.dstate, d.format, d.scale_block, work_fp32[l], stream);
             if (rc != SSDQ_OK) return rc;

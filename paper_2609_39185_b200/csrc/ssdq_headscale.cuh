@@ -124,7 +124,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_headscale_kernel(const Up
     thr.init(p.weyl, step_t, lis);
     const uint32_t key0 = (uint32_t)p.sr_seed, key1 = (uint32_t)(p.sr_seed >> 32);
     const uint32_t hash_base = step_t * kHashP2 + p.layer * kHashP3 + key0 * kHashP4;
-    const uint64_t grow_first = row_first + (uint64_t)p.batch_base * p.H * (NSLOT * RPS);
+    const uint64_t grow_first = row_first + p.row_off0 + (uint64_t)b * p.row_skip;
     uint32_t acc_row = 0;
     uint64_t grp_row = 0;
     if constexpr (RULE == RULE_WEYL) acc_row = thr.weyl_acc0(grow_first);

@@ -44,7 +44,9 @@ struct UpdateParams {
     uint32_t step_t;
     const uint32_t* step_base;   // null, or a device word added to step_t (replayable graphs keep their step count there)
     uint32_t layer;
-    uint32_t batch_base;
+    // global row of local row (b, h, p) = local row + row_off0 + b * row_skip  (rows of the [B_global * H_global * P, N] view):
+    uint64_t row_off0;       // (batch_index_base * H_global + head_index_base) * P
+    uint32_t row_skip;       // (H_global - H) * P: rows of other head shards between two local sequences
     uint32_t spi;            // slots per (b, h) item inside a CTA (power of two)
     uint32_t items_per_cta;
     uint32_t rps;            // rows per slot
@@ -70,6 +72,8 @@ struct QuantParams {
     uint32_t step_t;
     uint32_t layer;
     uint64_t row_base;
+    uint64_t rows_per_seq;    // 0, or rows of one local sequence: global row = row_base + row + (row / rows_per_seq) * row_skip
+    uint32_t row_skip;
     WeylConst weyl;
     uint64_t sr_seed;
 };

@@ -70,7 +70,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_mamba1_kernel(const Updat
 
     for (uint32_t b = b_first; b < b_last; ++b) {
         const uint64_t row = (uint64_t)b * p.H + d;
-        const uint64_t grow = row + (uint64_t)p.batch_base * p.H;
+        const uint64_t grow = row + p.row_off0 + (uint64_t)b * p.row_skip;
         uint4* sp = reinterpret_cast<uint4*>(p.state) + row * CH;
         // debug builds: the row's vectors, its x / y / dt elements, its scale and the sequence's B and C
         bool mem_ok = SSDQ_RANGE_OK(p, DBG_STATE, row * CH, CH, state_vecs) && SSDQ_RANGE_OK(p, DBG_ROWS, row, 1, rows) &&

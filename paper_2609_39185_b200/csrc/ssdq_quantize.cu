@@ -65,7 +65,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantParams p)
                 else p.scales[row * (N / 16) + lis] = s;
             }
         }
-        const uint64_t grow = p.row_base + row;
+        const uint64_t grow = p.row_base + row + (p.rows_per_seq ? (row / p.rows_per_seq) * p.row_skip : 0ull);
         uint32_t g_lo = 0, g_hi = 0, acc0 = 0;
         if constexpr (RULE == RULE_WEYL) acc0 = thr.weyl_acc0(grow);
         if constexpr (RULE == RULE_SR_HASH) acc0 = thr.hash_key0(grow, p.step_t * kHashP2 + p.layer * kHashP3 + key0 * kHashP4, key1);

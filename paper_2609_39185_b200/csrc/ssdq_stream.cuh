@@ -128,10 +128,9 @@ __global__ void __launch_bounds__(kThreads, SSDQ_STREAM_MINB) ssd_update_stream_
     const uint32_t key0 = (uint32_t)p.sr_seed, key1 = (uint32_t)(p.sr_seed >> 32);
     const uint32_t hash_base = step_t * kHashP2 + p.layer * kHashP3 + key0 * kHashP4;
     const bool y_writer = (lis & (LPR / 4 - 1)) == 0;
-    uint64_t grow_first = row0 + (uint64_t)p.batch_base * p.H * ROWS;
-
     uint32_t b = first / p.H;
     uint32_t h = first - b * p.H;
+    uint64_t grow_first = row0 + p.row_off0 + (uint64_t)b * p.row_skip;
     f32x2 B2[EPL / 2], C2[EPL / 2];
     // scalars of the next item are fetched one iteration ahead
     float dt_next = __ldg(p.dt + first), A_next = __ldg(p.A + h), D_next = (p.D && lis == 0) ? __ldg(p.D + h) : 0.0f;
@@ -265,6 +264,7 @@ __global__ void __launch_bounds__(kThreads, SSDQ_STREAM_MINB) ssd_update_stream_
       }
       h = 0;
       ++b;
+      grow_first += p.row_skip;       // over the rows that other head shards hold
     }
     cp_async_wait<0>();
 }

@@ -235,7 +235,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_kernel(const UpdateParams
     const uint32_t hash_base = step_t * kHashP2 + p.layer * kHashP3 + key0 * kHashP4;
     const uint32_t p_first = sub * p.rps;                         // first row of this slot inside the item
     const uint64_t row_first = (uint64_t)item * p.P + p_first;    // local row index (this call's tensors)
-    const uint64_t grow_first = row_first + (uint64_t)p.batch_base * p.H * p.P;   // global row index
+    const uint64_t grow_first = row_first + p.row_off0 + (uint64_t)b * p.row_skip;   // global row index
     uint4* state = reinterpret_cast<uint4*>(p.state);
     const bool row_scale = Fmt<FMT>::kScaled && (p.scale_block == (uint32_t)N);
 
@@ -473,7 +473,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
     LaneThreshold<FMT, RULE, LPR> thr;
     thr.init(p.weyl, step_t, lis);
     const uint32_t key0 = (uint32_t)p.sr_seed, key1 = (uint32_t)(p.sr_seed >> 32);
-    const uint64_t grow_first = row_first + (uint64_t)p.batch_base * p.H * (NSLOT * RPS);
+    const uint64_t grow_first = row_first + p.row_off0 + (uint64_t)b * p.row_skip;
     uint32_t acc_row = 0;
     uint64_t grp_row = 0;
     const uint32_t hash_base = step_t * kHashP2 + p.layer * kHashP3 + key0 * kHashP4;

@@ -42,7 +42,7 @@ class UpdateDesc(ctypes.Structure):
                 ("x", _vp), ("dt", _vp), ("A", _vp), ("Bm", _vp), ("Cm", _vp), ("D", _vp),
                 ("a_per_state", _u32), ("y", _vp), ("rule", _i32), ("weyl", Weyl), ("sr_seed", _u64),
                 ("layer", _u32), ("batch_index_base", _u32), ("dt_bias", _vp), ("z", _vp), ("dt_softplus", _u32),
-                ("ngroups", _u32)]
+                ("ngroups", _u32), ("head_index_base", _u32), ("nheads_global", _u32)]
 
 
 class StepInputs(ctypes.Structure):
@@ -172,7 +172,8 @@ def thresholds_materialize(rule, n, step_t, *, weyl=None, sr_seed=0, layer=0, fi
 
 
 def make_desc(state, scales, fmt, *, A, D, rule, weyl=None, sr_seed=0, layer=0, scale_block=0, batch_index_base=0,
-              x=None, dt=None, Bm=None, Cm=None, y=None, dt_bias=None, dt_softplus=False, ngroups=1, z=None) -> UpdateDesc:
+              x=None, dt=None, Bm=None, Cm=None, y=None, dt_bias=None, dt_softplus=False, ngroups=1, z=None,
+              head_index_base=0, nheads_global=0) -> UpdateDesc:
     """Describe one layer's problem.  `state` is a CUDA tensor of shape [B, H, P, N] holding the codes
     (uint8 for E4M3, int16/uint16/float16/bfloat16 for the 16-bit formats, float32 for the FP32 twin)."""
     B, H, P, N = state.shape
@@ -187,6 +188,7 @@ def make_desc(state, scales, fmt, *, A, D, rule, weyl=None, sr_seed=0, layer=0, 
         d.weyl = weyl
     d.sr_seed, d.layer, d.batch_index_base = sr_seed, layer, batch_index_base
     d.dt_bias, d.z, d.dt_softplus, d.ngroups = _ptr(dt_bias), _ptr(z), int(bool(dt_softplus)), ngroups
+    d.head_index_base, d.nheads_global = head_index_base, nheads_global
     # keep the tensors alive as long as the descriptor
     d._keep = (state, scales, A, D, x, dt, Bm, Cm, y, dt_bias, z)
     return d

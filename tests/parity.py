@@ -40,11 +40,13 @@ class Pair:
     """One layer's state held twice: on the GPU (library) and on the host (oracle)."""
 
     def __init__(self, shape, fmt, rule, A, D, *, weyl_block=16, scale_block=0, layer=0, weyl_seed=0, sr_seed=0,
-                 batch_index_base=0, h0_codes=None, h0_scales=None, dt_bias=None, dt_softplus=False, ngroups=1):
+                 batch_index_base=0, h0_codes=None, h0_scales=None, dt_bias=None, dt_softplus=False, ngroups=1,
+                 head_index_base=0, nheads_global=0):
         self.shape, self.fmt, self.rule = shape, fmt, rule
         self.A, self.D = A, D
         self.kw = dict(layer=layer, weyl_seed=weyl_seed, weyl_block=weyl_block, sr_seed=sr_seed,
-                       batch_index_base=batch_index_base, dt_bias=dt_bias, dt_softplus=dt_softplus, ngroups=ngroups)
+                       batch_index_base=batch_index_base, dt_bias=dt_bias, dt_softplus=dt_softplus, ngroups=ngroups,
+                       head_index_base=head_index_base, nheads_global=nheads_global)
         self.bias_d = to_dev(dt_bias)
         self.scale_block = scale_block
         if h0_codes is None:
@@ -59,7 +61,7 @@ class Pair:
         self.desc = ssdq.make_desc(self.state_d, self.scales_d, fmt, A=self.A_d, D=self.D_d, rule=rule, weyl=weyl,
                                    sr_seed=sr_seed, layer=layer, scale_block=scale_block,
                                    batch_index_base=batch_index_base, dt_bias=self.bias_d, dt_softplus=dt_softplus,
-                                   ngroups=ngroups)
+                                   ngroups=ngroups, head_index_base=head_index_base, nheads_global=nheads_global)
         self.y_d = torch.empty(shape[:3], dtype=torch.float32, device="cuda")
 
     def step_gpu(self, t, x, dt, Bm, Cm, z=None):

@@ -34,7 +34,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 def test_struct_sizes_match_the_header():
     assert ctypes.sizeof(ssdq.Weyl) == 32
-    assert ctypes.sizeof(ssdq.UpdateDesc) == 184
+    assert ctypes.sizeof(ssdq.UpdateDesc) == 192
     assert ctypes.sizeof(ssdq.StepInputs) == 104
 
 
@@ -73,6 +73,9 @@ def _desc(**over):
     (dict(format=ssdq.E4M3, scales=0x20000, scale_block=8 * 128), ssdq.ERR_UNSUPPORTED),
     (dict(format=ssdq.FP32, dstate=256), ssdq.ERR_UNSUPPORTED),
     (dict(weyl=ssdq.Weyl()), ssdq.ERR_SHAPE),
+    (dict(head_index_base=1), ssdq.ERR_SHAPE),                       # a head offset needs nheads_global
+    (dict(head_index_base=1, nheads_global=4), ssdq.ERR_SHAPE),      # heads 1..4 of 4
+    (dict(nheads_global=3), ssdq.ERR_SHAPE),                         # fewer heads in the layer than in the call
 ])
 def test_bad_arguments_are_rejected_before_any_launch(lib, over, status):
     before = ssdq.launch_count()

@@ -546,3 +546,102 @@ def test_graph_replay_on_the_persistent_kernel():
         assert torch.equal(s1[l], s2[l]) and torch.equal(c1[l], c2[l])
     assert torch.equal(y1, y2)
     graph.close()
+
+
+HEAD_SHARD_CASES = [
+    # fmt, (B, H_global, P, N), per-state A, scale granularity, kernel family the shard runs on
+    (ssdq.BF16, (3, 6, 64, 128), False, None, "ssd_update_tile_kernel"),
+    (ssdq.FP16, (3, 6, 64, 64), False, None, "ssd_update_tile_kernel"),
+    (ssdq.E4M3, (3, 6, 64, 128), False, "row", "ssd_update_stream_kernel"),
+    (ssdq.INT8, (3, 6, 128, 128), False, "block16", "ssd_update_stream_kernel"),
+    (ssdq.E4M3, (3, 6, 64, 128), False, "head", "ssd_update_headscale_kernel"),
+    (ssdq.BF16, (5, 96, 1, 16), True, None, "ssd_update_mamba1_kernel"),
+    (ssdq.INT8, (5, 96, 1, 16), True, "row", "ssd_update_mamba1_kernel"),
+    (ssdq.BF16, (3, 6, 8, 32), True, None, "ssd_update_kernel"),
+]
+
+
+@pytest.mark.parametrize("rule", [ssdq.WEYL, ssdq.SR, ssdq.SR_HASH])
+@pytest.mark.parametrize("fmt,shape,aps,scale,family", HEAD_SHARD_CASES)
+def test_a_head_shard_reproduces_the_bits_of_the_whole_layer(fmt, shape, aps, scale, family, rule):
+    """Tensor-parallel split: a call that holds heads [h0, h1) of the layer, told head_index_base = h0 and
+    nheads_global = H, writes the codes that the unsharded call writes for those heads (the thresholds of Eq. 2 are
+    drawn at the entry's index in the whole layer: Appendix B "Dithers" numbers the rows of the full state matrix).
+    Checked against the oracle on the shard and against the library's own unsharded run, with a batch offset on top."""
+    B, Hg, P, N = shape
+    f32 = np.float32
+    rng = np.random.default_rng(hash((fmt, shape, aps)) % 2**31)
+    sb = {None: 0, "row": N, "block16": 16, "head": P * N}[scale]
+    A = (-np.exp(rng.uniform(-3, 1, (Hg, N) if aps else Hg))).astype(f32)
+    D = rng.normal(0, 0.1, Hg).astype(f32)
+    wb = 16
+    bbase = 7
+    whole = Pair((B, Hg, P, N), fmt, rule, A, D, weyl_block=wb, scale_block=sb, layer=3, weyl_seed=2, sr_seed=11, batch_index_base=bbase)
+    h0 = Hg // 3
+    h1 = Hg - Hg // 6
+    part = Pair((B, h1 - h0, P, N), fmt, rule, A[h0:h1].copy(), D[h0:h1].copy(), weyl_block=wb, scale_block=sb, layer=3, weyl_seed=2,
+                sr_seed=11, batch_index_base=bbase, head_index_base=h0, nheads_global=Hg)
+    for t in range(1, 5):
+        x = rng.standard_normal((B, Hg, P)).astype(f32)
+        dt = np.log1p(np.exp(rng.normal(-2, 0.5, (B, Hg)))).astype(f32)
+        Bm = (rng.standard_normal((B, N)) / np.sqrt(N)).astype(f32)
+        Cm = rng.standard_normal((B, N)).astype(f32)
+        whole.step_gpu(t, x, dt, Bm, Cm)
+        xs, dts = np.ascontiguousarray(x[:, h0:h1]), np.ascontiguousarray(dt[:, h0:h1])
+        part.step_gpu(t, xs, dts, Bm, Cm)
+        assert ssdq.last_kernel() == family
+        y_ref = part.step_oracle(t, xs, dts, Bm, Cm)
+        part.compare(t, xs, dts, Bm, Cm, y_ref)
+        assert np.array_equal(codes_to_host(part.state_d, fmt), codes_to_host(whole.state_d, fmt)[:, h0:h1]), t
+        if part.scales_d is not None:
+            ws = whole.scales_d.cpu().numpy().reshape(B, Hg, -1)[:, h0:h1]
+            assert np.array_equal(part.scales_d.cpu().numpy().reshape(B, h1 - h0, -1), ws), t
+        assert np.array_equal(part.y_d.cpu().numpy(), whole.y_d.cpu().numpy()[:, h0:h1]), t
+
+
+def test_head_shard_arguments_are_checked():
+    st = torch.zeros((2, 4, 16, 64), dtype=torch.int16, device="cuda")
+    A = torch.zeros(4, device="cuda")
+    x = torch.zeros((2, 4, 16), device="cuda"); dt = torch.zeros((2, 4), device="cuda"); Bm = torch.zeros((2, 64), device="cuda")
+    for hb, hg in ((1, 0), (1, 4), (0, 3), (5, 8)):
+        d = ssdq.make_desc(st, None, ssdq.BF16, A=A, D=None, rule=ssdq.RTN, head_index_base=hb, nheads_global=hg)
+        with pytest.raises(ssdq.SsdqError) as e:
+            ssdq.ssd_state_update(d, 1, x=x, dt=dt, Bm=Bm, Cm=Bm, y=torch.empty_like(x))
+        assert e.value.status == ssdq.ERR_SHAPE
+    d = ssdq.make_desc(st, None, ssdq.BF16, A=A, D=None, rule=ssdq.RTN, head_index_base=4, nheads_global=8)
+    ssdq.ssd_state_update(d, 1, x=x, dt=dt, Bm=Bm, Cm=Bm, y=torch.empty_like(x))
+
+
+@pytest.mark.parametrize("fmt", [ssdq.BF16, ssdq.INT8])
+@pytest.mark.parametrize("rule", [ssdq.WEYL, ssdq.SR])
+def test_checkpointed_rounding_on_a_head_shard(fmt, rule):
+    """The checkpointing driver rounds a head shard's rows at their indices in the whole layer: heads 1..2 of 4, every
+    second write rounded, equal the same heads of the unsharded checkpointed run."""
+    from dataclasses import replace
+    cfg = replace(workloads.CONFIGS[4], batch=3, nheads=4, fmt=fmt)
+    sb, wb = (cfg.scale_block if oracle.has_block_scale(fmt) else 0), cfg.weyl_block
+    T, h0, h1 = 6, 1, 3
+    A, D = workloads.layer_params(cfg)
+    ins = [workloads.step_inputs(cfg, t) for t in range(1, T + 1)]
+    stack = lambda i, sl: to_dev(np.stack([np.ascontiguousarray(ins[t][i][:, sl] if i < 2 else ins[t][i])[None] for t in range(T)]))
+
+    def run(sl, **shard):
+        nh = len(range(*sl.indices(cfg.nheads)))
+        shape = (cfg.batch, nh) + cfg.state_shape[2:]
+        st_h, sc_h = oracle.new_state(shape, fmt, sb)
+        st, sc = codes_to_dev(st_h, fmt), to_dev(sc_h)
+        desc = ssdq.make_desc(st, sc, fmt, A=to_dev(A[sl].copy()), D=to_dev(D[sl].copy()), rule=rule,
+                              weyl=ssdq.weyl_offsets_init(0, 0, wb), sr_seed=1, scale_block=sb, batch_index_base=5, **shard)
+        xs, dts, Bs, Cs = (stack(i, sl) for i in range(4))
+        y = torch.zeros_like(xs)
+        work = torch.zeros(shape, dtype=torch.float32, device="cuda")
+        ssdq.ssd_decode_run_checkpointed([desc], [work], 2, 1, T, ssdq.make_step_inputs(xs, dts, Bs, Cs, y))
+        torch.cuda.synchronize()
+        return st, sc, y
+
+    st_w, sc_w, y_w = run(slice(0, cfg.nheads))
+    st_p, sc_p, y_p = run(slice(h0, h1), head_index_base=h0, nheads_global=cfg.nheads)
+    assert torch.equal(st_p, st_w[:, h0:h1])
+    if sc_w is not None:
+        assert torch.equal(sc_p.reshape(cfg.batch, h1 - h0, -1), sc_w.reshape(cfg.batch, cfg.nheads, -1)[:, h0:h1])
+    assert torch.equal(y_p, y_w[:, :, :, h0:h1])

@@ -178,6 +178,8 @@ def test_update_against_python_restatement_on_tiny_state(fmt, rule, a_per_state)
     A = -np.exp(rng.uniform(-3, 1, (H, N) if a_per_state else (H,))).astype(f32)
     D = rng.normal(0, 0.1, H).astype(f32)
     base = 3
+    # half of the cases hold heads 2..4 of a layer with 7 heads: the entry index counts the heads that are not here
+    hb, Hg = (2, 7) if a_per_state else (0, H)
     for t in (1, 2, 3):
         x = rng.standard_normal((Bsz, H, P)).astype(f32)
         dt = np.log1p(np.exp(rng.normal(-2, 0.5, (Bsz, H)))).astype(f32)
@@ -211,7 +213,7 @@ def test_update_against_python_restatement_on_tiny_state(fmt, rule, a_per_state)
                             want_scales[(((b * H + h) * P + p) * N + k0) // 16] = s
                         for j in range(16):
                             n = k0 + j
-                            flat = ((((base + b) * H + h) * P + p) * N + n)
+                            flat = ((((base + b) * Hg + hb + h) * P + p) * N + n)
                             if rule == WEYL:
                                 U = oracle.weyl_u24(flat // wb, flat % wb, 2, 1, t)
                             elif rule == SR:
@@ -225,7 +227,8 @@ def test_update_against_python_restatement_on_tiny_state(fmt, rule, a_per_state)
                             if q == 0.0 and np.signbit(v):
                                 want_codes[b, h, p, n] = oracle.encode(f32(-0.0), fmt)[0]
         y = oracle.state_update(state, sc, fmt, sb, x, dt, A, Bm, Cm, D, rule, t, layer=2, weyl_seed=1,
-                                weyl_block=wb, sr_seed=9, batch_index_base=base)
+                                weyl_block=wb, sr_seed=9, batch_index_base=base, head_index_base=hb,
+                                nheads_global=Hg if a_per_state else 0)
         assert np.array_equal(state, want_codes)
         if sc is not None:
             assert np.array_equal(sc, want_scales)
@@ -245,6 +248,19 @@ def test_sharding_invariance_of_indices():
             y2 = oracle.state_update(part, None, FP16, 0, x[2:], dt[2:], A, Bm[2:], Cm[2:], D, rule, t,
                                      batch_index_base=2)
             assert np.array_equal(full[2:], part) and np.array_equal(y[2:], y2)
+    # a head slice with head_index_base and the layer's head count does the same (every sequence, heads 1..2 of 4)
+    for rule in (SR, WEYL):
+        full, _ = oracle.new_state(cfg.state_shape, FP16)
+        part = np.ascontiguousarray(full[:, 1:3])
+        for t in range(1, 6):
+            x, dt, Bm, Cm = workloads.step_inputs(cfg, t)
+            y = oracle.state_update(full, None, FP16, 0, x, dt, A, Bm, Cm, D, rule, t)
+            y2 = oracle.state_update(part, None, FP16, 0, np.ascontiguousarray(x[:, 1:3]), np.ascontiguousarray(dt[:, 1:3]),
+                                     A[1:3].copy(), Bm, Cm, D[1:3].copy(), rule, t, head_index_base=1, nheads_global=4)
+            assert np.array_equal(full[:, 1:3], part) and np.array_equal(y[:, 1:3], y2)
+    with pytest.raises(ValueError):
+        oracle.state_update(part, None, FP16, 0, np.ascontiguousarray(x[:, 1:3]), np.ascontiguousarray(dt[:, 1:3]),
+                            A[1:3].copy(), Bm, Cm, D[1:3].copy(), WEYL, 1, head_index_base=3, nheads_global=4)
 
 
 # ---- the rest of a production signature: dt_bias + softplus, grouped B/C, z gate -----------------

@@ -1,5 +1,6 @@
 """The N > 1 mode on CPU: two gloo ranks each run the oracle on their batch shard with the shard's
-global batch base; together they reproduce the unsharded run bit for bit, and timings reduce by max."""
+global batch base, then on their head shard with its head base; either way they reproduce the unsharded
+run bit for bit together, and timings reduce by max."""
 import os
 import sys
 
@@ -29,8 +30,20 @@ def _worker(rank, world, port, out):
             x, dt, Bm, Cm = workloads.step_inputs(cfg, t, batch_slice=sl)
             oracle.state_update(st, None, cfg.fmt, 0, x, dt, A, Bm, Cm, D, rule, t, batch_index_base=base)
         results[rule] = st
+    # the same layer split over the heads instead (tensor parallel): every sequence, this rank's heads
+    from paper_2609_39185_b200.replicas import shard_head_range
+    h0, h1 = shard_head_range(rank, world, cfg.nheads)
+    heads = {}
+    for rule in (oracle.SR, oracle.WEYL):
+        st, _ = oracle.new_state((cfg.batch, h1 - h0) + cfg.state_shape[2:], cfg.fmt)
+        for t in range(1, 9):
+            x, dt, Bm, Cm = workloads.step_inputs(cfg, t)
+            oracle.state_update(st, None, cfg.fmt, 0, np.ascontiguousarray(x[:, h0:h1]), np.ascontiguousarray(dt[:, h0:h1]),
+                                A[h0:h1].copy(), Bm, Cm, D[h0:h1].copy(), rule, t, head_index_base=h0, nheads_global=cfg.nheads)
+        heads[rule] = st
     slowest = max_over_ranks(1.0 + rank, dist)
-    np.savez(os.path.join(out, f"rank{rank}.npz"), sr=results[oracle.SR], weyl=results[oracle.WEYL], slowest=slowest)
+    np.savez(os.path.join(out, f"rank{rank}.npz"), sr=results[oracle.SR], weyl=results[oracle.WEYL], slowest=slowest,
+             sr_heads=heads[oracle.SR], weyl_heads=heads[oracle.WEYL])
     dist.barrier()
     dist.destroy_process_group()
 
@@ -50,4 +63,5 @@ def test_two_replicas_equal_one_big_batch(tmp_path):
             oracle.state_update(full, None, cfg.fmt, 0, x, dt, A, Bm, Cm, D, rule, t)
         parts = [np.load(os.path.join(tmp_path, f"rank{r}.npz")) for r in range(world)]
         assert np.array_equal(np.concatenate([p[name] for p in parts]), full)
+        assert np.array_equal(np.concatenate([p[name + "_heads"] for p in parts], axis=1), full)
         assert all(float(p["slowest"]) == 2.0 for p in parts)
