@@ -273,6 +273,15 @@ const char* ssdq_last_kernel(void);
  * of the library on the same thread. */
 const char* ssdq_last_error(void);
 
+/* Launch overlap inside the multi-launch stream drivers (ssd_decode_run, ssd_decode_run_checkpointed): when enabled
+ * (the default) every fused-update launch after the first of a call carries the programmatic-stream-serialization attribute, so its CTAs are scheduled while the previous kernel of the driver drains;
+ * each kernel waits for the completion of all earlier grids before it touches memory, so results do not change (the
+ * paper has no counterpart: this is launch plumbing).  The drivers' inputs must not be written by other work while a
+ * driver call is in flight, which the drivers require anyway.  A single ssd_state_update call never uses the attribute.
+ * Graphs are captured without it (plain edges replay faster) and ssd_decode_run_host launches without it (it was
+ * measured to lose beside the copy streams).  Returns the previous setting.  Process-wide. */
+int ssdq_set_launch_overlap(int enabled);
+
 /* Number of kernels the library has launched in this process (a counter for benchmarks). */
 uint64_t ssdq_launch_count(void);
 

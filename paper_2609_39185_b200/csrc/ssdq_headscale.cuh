@@ -13,6 +13,7 @@ namespace ssdq {
 
 template <int FMT, int RULE, int LPR, int RPS>
 __global__ void __launch_bounds__(kThreads) ssd_update_headscale_kernel(const UpdateParams p) {
+    grid_dependency_gate(p.overlap);
     static_assert(Fmt<FMT>::kScaled && Fmt<FMT>::kEpl == 16, "one-byte block-scaled stores");
     constexpr int EPL = 16;
     constexpr int N = LPR * EPL;
@@ -21,7 +22,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_headscale_kernel(const Up
     constexpr int GRP = RPS >= 4 ? 4 : 2;
     static_assert(RPS % GRP == 0 && LPR >= GRP && RPS <= 8, "rows are reduced GRP at a time; at most 8 rows per lane stay in registers");
 
-    const uint32_t step_t = p.step_t + (p.step_base ? __ldg(p.step_base) : 0u);
+    const uint32_t step_t = p.step_t + (p.step_base ? __ldcg(p.step_base) : 0u);
     const uint32_t lis = threadIdx.x % LPR;
     const uint32_t slot = threadIdx.x / LPR;
     const uint32_t h = blockIdx.x, b = blockIdx.y;
@@ -158,8 +159,7 @@ cudaError_t try_launch_headscale(const UpdateParams& p, cudaStream_t stream, boo
             launched = true;                                                                       \
             note_kernel(3);                                                                        \
             if (p.prepare_only) return cudaSuccess;                                                \
-            ssd_update_headscale_kernel<FMT, RULE, LPR, R><<<grid, kThreads, 0, stream>>>(p);      \
-            return cudaGetLastError();                                                             \
+            return launch_update_kernel(ssd_update_headscale_kernel<FMT, RULE, LPR, R>, grid, 0, stream, p); \
         }
         SSDQ_HEAD_CASE(4u)
         SSDQ_HEAD_CASE(8u)

@@ -52,6 +52,7 @@ struct UpdateParams {
     uint32_t rps;            // rows per slot
     WeylConst weyl;
     uint64_t sr_seed;
+    uint32_t overlap;        // 0: plain launch; else programmatic stream serialization: 1 wait, then release the successor; 2 release first
     uint32_t prepare_only;   // host side only: pick the kernel and do its one-time set-up (attributes, occupancy), launch nothing
 #ifdef SSDQ_DEBUG
     DebugBounds dbg;

@@ -41,16 +41,33 @@ __device__ __forceinline__ f32x2 exp_spec2(f32x2 z2) {
 
 // grid = (ceil(H / kThreads), batch chunks); CTA (cx, cy) owns channels cx * kThreads .. and sequences
 // [cy * b_per_cta, (cy + 1) * b_per_cta).  N = 16, P = 1, A is [H, 16].
+//
+// A lane works on one row at a time and a row is a long dependent computation, so the bytes of the NEXT row (its codes,
+// dt, x, scale, and the sequence's B and C) are requested with asynchronous copies into a two-stage shared-memory ring
+// before the current row is computed: the loads cost no registers and their latency hides behind the arithmetic.
+// Each lane copies its own row; B and C of a sequence (128 bytes, the same for the whole warp) are copied once per warp
+// by its first eight lanes.  Channels beyond H (last tile only) run on a clamped channel and store nothing.
+// With the loads out of the way the kernel is bound by instruction issue (every entry needs its own exponential), so
+// the dithered rules, which need more registers, trade two resident CTAs for a spill-free loop (measured).
 template <int FMT, int RULE>
-__global__ void __launch_bounds__(kThreads) ssd_update_mamba1_kernel(const UpdateParams p) {
+__global__ void __launch_bounds__(kThreads, RULE == RULE_RTN ? 8 : 6) ssd_update_mamba1_kernel(const UpdateParams p) {
+    grid_dependency_gate(p.overlap);
     constexpr int EPL = Fmt<FMT>::kEpl;                 // entries per 16-byte chunk: 8 (two-byte codes) or 16
     constexpr int N = 16;
     constexpr int CH = N / EPL;                         // chunks per row: 2 or 1
-    const uint32_t step_t = p.step_t + (p.step_base ? __ldg(p.step_base) : 0u);
-    const uint32_t d = blockIdx.x * kThreads + threadIdx.x;
-    if (d >= p.H) return;                               // no block-wide operation follows
+    constexpr unsigned FULL = 0xFFFFFFFFu;
+    __shared__ __align__(16) uint4 s_codes[2][CH][kThreads];
+    __shared__ __align__(16) float s_bc[2][kThreads / 32][2 * N];     // per warp: B[0..15], C[0..15] of the sequence
+    __shared__ float s_dt[2][kThreads], s_x[2][kThreads], s_sc[2][kThreads];
+
+    const uint32_t step_t = p.step_t + (p.step_base ? __ldcg(p.step_base) : 0u);
+    const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+    const uint32_t d_raw = blockIdx.x * kThreads + tid;
+    const bool active = d_raw < p.H;
+    const uint32_t d = active ? d_raw : p.H - 1u;
     const uint32_t b_first = blockIdx.y * p.rps;        // rps: sequences per CTA
     const uint32_t b_last = min(b_first + p.rps, p.B);
+    if (b_first >= b_last) return;                      // the whole CTA
 
     f32x2 A2[N / 2];
     {
@@ -68,23 +85,55 @@ __global__ void __launch_bounds__(kThreads) ssd_update_mamba1_kernel(const Updat
     // Weyl: a row is one dither block (block 16 = N): r = global row, c = n
     const uint32_t weyl_const = p.weyl.mul_row + p.weyl.mul_col + p.weyl.base + step_t * p.weyl.phi;
 
-    for (uint32_t b = b_first; b < b_last; ++b) {
+    const uint32_t codes_s = (uint32_t)__cvta_generic_to_shared(&s_codes[0][0][tid]);     // + stage * CH * kThreads * 16 + c * kThreads * 16
+    const uint32_t dt_s = (uint32_t)__cvta_generic_to_shared(&s_dt[0][tid]);              // + stage * kThreads * 4
+    const uint32_t x_s = (uint32_t)__cvta_generic_to_shared(&s_x[0][tid]);
+    const uint32_t sc_s = (uint32_t)__cvta_generic_to_shared(&s_sc[0][tid]);
+    const uint32_t bc_s = (uint32_t)__cvta_generic_to_shared(&s_bc[0][warp][(lane & 7u) * 4u]);   // + stage * sizeof(s_bc[0])
+    uint32_t ok_bits = 0;                               // bit s: the row in stage s passed the debug build's range checks
+    auto issue = [&](uint32_t b, uint32_t stage) {
+        const uint64_t row = (uint64_t)b * p.H + d;
+        // debug builds: the row's vectors, its x / y / dt elements, its scale and the sequence's B and C
+        bool ok = SSDQ_RANGE_OK(p, DBG_STATE, row * CH, CH, state_vecs) && SSDQ_RANGE_OK(p, DBG_ROWS, row, 1, rows) &&
+                  SSDQ_RANGE_OK(p, DBG_ITEMS, row, 1, items) && SSDQ_RANGE_OK(p, DBG_BC, (size_t)b * N, N, bc_floats);
+        if constexpr (Fmt<FMT>::kScaled) ok = ok && SSDQ_RANGE_OK(p, DBG_SCALES, row, 1, scales);
+#ifdef SSDQ_DEBUG
+        ok = __all_sync(FULL, ok);                      // lanes copy one another's rows and meet at warp barriers: skip as a warp
+#endif
+        ok_bits = (ok_bits & ~(1u << stage)) | ((uint32_t)ok << stage);
+        if (!ok) return;
+        // .ca: a two-byte row is two 16-byte chunks 32 bytes apart per lane, so each copy instruction touches every
+        // sector of the warp's kilobyte; keeping the lines in L1 lets the second one hit there
+        const uint4* sp = reinterpret_cast<const uint4*>(p.state) + row * CH;
+#pragma unroll
+        for (int c = 0; c < CH; ++c) cp_async16_ca(codes_s + (stage * CH + c) * (kThreads * 16u), sp + c);
+        cp_async4_ca(dt_s + stage * (kThreads * 4u), p.dt + row);
+        cp_async4_ca(x_s + stage * (kThreads * 4u), p.x + row);
+        if constexpr (Fmt<FMT>::kScaled) cp_async4_ca(sc_s + stage * (kThreads * 4u), p.scales + row);
+        if (lane < 8u) cp_async16_ca(bc_s + stage * (uint32_t)sizeof(s_bc[0]), (lane < 4u ? p.Bm : p.Cm) + (size_t)b * N + (lane & 3u) * 4u);
+    };
+    issue(b_first, 0u);
+    cp_async_commit();
+
+    uint32_t stage = 0;
+    for (uint32_t b = b_first; b < b_last; ++b, stage ^= 1u) {
+        __syncwarp(FULL);                               // every lane is done with the B / C of the stage refilled next
+        if (b + 1 < b_last) issue(b + 1, stage ^ 1u);
+        cp_async_commit();
+        cp_async_wait<1>();                             // this row's group has landed (the next one may be pending)
+        __syncwarp(FULL);                               // ... also the B / C chunks that other lanes copied
+        if (!((ok_bits >> stage) & 1u)) continue;                 // debug builds only, and then the whole warp
         const uint64_t row = (uint64_t)b * p.H + d;
         const uint64_t grow = row + p.row_off0 + (uint64_t)b * p.row_skip;
         uint4* sp = reinterpret_cast<uint4*>(p.state) + row * CH;
-        // debug builds: the row's vectors, its x / y / dt elements, its scale and the sequence's B and C
-        bool mem_ok = SSDQ_RANGE_OK(p, DBG_STATE, row * CH, CH, state_vecs) && SSDQ_RANGE_OK(p, DBG_ROWS, row, 1, rows) &&
-                      SSDQ_RANGE_OK(p, DBG_ITEMS, row, 1, items) && SSDQ_RANGE_OK(p, DBG_BC, (size_t)b * N, N, bc_floats);
-        if constexpr (Fmt<FMT>::kScaled) mem_ok = mem_ok && SSDQ_RANGE_OK(p, DBG_SCALES, row, 1, scales);
-        if (!mem_ok) continue;          // a lane on its own: nothing below involves another thread
         uint4 raw[CH];
 #pragma unroll
-        for (int c = 0; c < CH; ++c) raw[c] = sp[c];
-        const float dtv = __ldg(p.dt + row), xv = __ldg(p.x + row);
+        for (int c = 0; c < CH; ++c) raw[c] = s_codes[stage][c][tid];
+        const float dtv = s_dt[stage][tid], xv = s_x[stage][tid];
         float sc_old = 0.0f;
-        if constexpr (Fmt<FMT>::kScaled) sc_old = p.scales[row];
-        const float4* Bp = reinterpret_cast<const float4*>(p.Bm + (size_t)b * N);
-        const float4* Cp = reinterpret_cast<const float4*>(p.Cm + (size_t)b * N);
+        if constexpr (Fmt<FMT>::kScaled) sc_old = s_sc[stage][tid];
+        const float4* Bp = reinterpret_cast<const float4*>(&s_bc[stage][warp][0]);       // the same address in every lane: a broadcast
+        const float4* Cp = Bp + N / 4;
         const float dtx = __fmul_rn(dtv, xv);
         const f32x2 dt2 = pack2(dtv, dtv), dtx2 = pack2(dtx, dtx), sc2 = pack2(sc_old, sc_old);
         float hin[N];
@@ -95,7 +144,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_mamba1_kernel(const Updat
         float amax = 0.0f;
 #pragma unroll
         for (int i = 0; i < N / 4; ++i) {
-            const float4 bb = __ldg(Bp + i), cc = __ldg(Cp + i);       // the same address in every lane: a broadcast
+            const float4 bb = Bp[i], cc = Cp[i];
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
                 const int q = 2 * i + j;
@@ -114,7 +163,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_mamba1_kernel(const Updat
                 }
             }
         }
-        {
+        if (active) {
             float d0, d1;
             unpack2(dot2, d0, d1);
             p.y[row] = __fadd_rn(d0, d1);
@@ -126,7 +175,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_mamba1_kernel(const Updat
             const f32x2 rinv2 = pack2(rinv, rinv);
 #pragma unroll
             for (int q = 0; q < N / 2; ++q) unpack2(mul2_rn(hn[q], rinv2), v[2 * q], v[2 * q + 1]);
-            p.scales[row] = s;
+            if (active) p.scales[row] = s;
         } else {
 #pragma unroll
             for (int q = 0; q < N / 2; ++q) unpack2(hn[q], v[2 * q], v[2 * q + 1]);
@@ -141,10 +190,12 @@ __global__ void __launch_bounds__(kThreads) ssd_update_mamba1_kernel(const Updat
             uint32_t acc0 = acc_row;
             if constexpr (RULE == RULE_WEYL) acc0 = acc_row + (uint32_t)(c * EPL) * p.weyl.mul_col;
             if constexpr (RULE == RULE_SR_HASH) acc0 = acc_row + (uint32_t)(c * EPL) * kHashP1;
-            sp[c] = round_pack_lane<FMT, RULE>(v + c * EPL, acc0, p.weyl.mul_col, (uint32_t)g, (uint32_t)(g >> 32), step_t, p.layer,
-                                               key0, key1, p.scale_top);
+            const uint4 packed = round_pack_lane<FMT, RULE>(v + c * EPL, acc0, p.weyl.mul_col, (uint32_t)g, (uint32_t)(g >> 32), step_t, p.layer,
+                                                            key0, key1, p.scale_top);
+            if (active) sp[c] = packed;
         }
     }
+    cp_async_wait<0>();
 }
 
 // Shapes covered: N = 16, headdim 1, one decay per state, the plain signature, scale and dither blocks of 16.
@@ -167,8 +218,7 @@ cudaError_t try_launch_mamba1(const UpdateParams& p, cudaStream_t stream, bool& 
         launched = true;
         note_kernel(4);
         if (p.prepare_only) return cudaSuccess;
-        ssd_update_mamba1_kernel<FMT, RULE><<<dim3(tiles, chunks), kThreads, 0, stream>>>(q);
-        return cudaGetLastError();
+        return launch_update_kernel(ssd_update_mamba1_kernel<FMT, RULE>, dim3(tiles, chunks), 0, stream, q);
     }
     return cudaSuccess;
 }

@@ -36,19 +36,6 @@ __device__ __forceinline__ void unpack4_int8_x2(uint32_t w, f32x2& p01, f32x2& p
     p23 = add2_rn(pack2u(__byte_perm(w, 0x4B000000u, 0x7542), __byte_perm(w, 0x4B000000u, 0x7543)), off);
 }
 
-__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gmem_src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void cp_async16_ca(uint32_t smem_dst, const void* gmem_src) {
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void cp_async4_ca(uint32_t smem_dst, const void* gmem_src) {
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int PENDING>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory"); }
-
 // Shared memory of one CTA: STAGES x { codes [RPS][kThreads] x 16 B, x [RPS/4][kThreads] x 16 B, scales [RPS/4][kThreads] x 16 B }.
 template <int RPS, int STAGES>
 constexpr size_t stream_smem_bytes() { return (size_t)STAGES * kThreads * 16u * (RPS + 2 * (RPS / 4)); }
@@ -58,6 +45,7 @@ constexpr size_t stream_smem_bytes() { return (size_t)STAGES * kThreads * 16u * 
 // grid = any number of CTAs <= n_items; CTA c owns items [c n / G, (c + 1) n / G).
 template <int FMT, int RULE, int LPR, int RPS, int STAGES, bool ROW_SCALE>
 __global__ void __launch_bounds__(kThreads, SSDQ_STREAM_MINB) ssd_update_stream_kernel(const UpdateParams p) {
+    grid_dependency_gate(p.overlap);
     static_assert(Fmt<FMT>::kScaled && Fmt<FMT>::kEpl == 16, "one-byte block-scaled stores");
     static_assert(RPS % 4 == 0 && LPR >= 4 && STAGES >= 2, "rows are processed four at a time");
     constexpr int EPL = 16;
@@ -81,7 +69,7 @@ __global__ void __launch_bounds__(kThreads, SSDQ_STREAM_MINB) ssd_update_stream_
     const uint32_t first = (uint32_t)(((uint64_t)blockIdx.x * p.n_items) / gridDim.x);
     const uint32_t last = (uint32_t)(((uint64_t)(blockIdx.x + 1) * p.n_items) / gridDim.x);
     if (first >= last) return;
-    const uint32_t step_t = p.step_t + (p.step_base ? __ldg(p.step_base) : 0u);
+    const uint32_t step_t = p.step_t + (p.step_base ? __ldcg(p.step_base) : 0u);
     const float top = p.scale_top, inv_top = p.inv_scale_top;
 
     // pointers of the item being fetched (f_*) and of the item being computed (c_*), advanced by one item per iteration
@@ -304,8 +292,7 @@ inline cudaError_t launch_stream(const UpdateParams& p, cudaStream_t stream) {
     if (grid > p.n_items) grid = p.n_items;
     note_kernel(2);
     if (p.prepare_only) return cudaSuccess;
-    ssd_update_stream_kernel<FMT, RULE, LPR, RPS, STAGES, ROW_SCALE><<<grid, kThreads, stream_smem_bytes<RPS, STAGES>(), stream>>>(p);
-    return cudaGetLastError();
+    return launch_update_kernel(ssd_update_stream_kernel<FMT, RULE, LPR, RPS, STAGES, ROW_SCALE>, dim3(grid), stream_smem_bytes<RPS, STAGES>(), stream, p);
 }
 
 // Shapes covered: N = 128 with heads of 64 or 128 rows, the plain signature (no dt_bias / softplus / groups / gate),

@@ -141,6 +141,53 @@ __device__ __forceinline__ uint4 round_pack_lane(const float* v, uint32_t acc0, 
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
+// Asynchronous global -> shared copies (cg: through L2 only; ca: also kept in L1), grouped by commit.
+__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async16_ca(uint32_t smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async4_ca(uint32_t smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int PENDING>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory"); }
+
+// Programmatic dependent launch.  Every fused-update kernel opens with grid_dependency_gate(): it waits until every
+// earlier grid of the stream has completed and its writes are visible -- before the kernel touches any memory -- and
+// lets the next kernel of the stream be scheduled, so that kernel's launch latency and CTA ramp overlap this one's
+// execution.  The data dependency between the steps of a layer is kept by the wait (each kernel waits for its
+// predecessor, which waited for its own, so completion is transitive).  Order of the two: a grid of many waves releases
+// its successor first (the successor's CTAs can only become resident in the last wave anyway, and they are then in place
+// when the tail drains); a small grid waits first, because releasing first lets waiting CTAs of several later launches
+// pile up beside the running ones, which was measured to slow small launches down.  Launched without the attribute the
+// two instructions do nothing.
+__device__ __forceinline__ void grid_dependency_gate(uint32_t mode) {
+    if (mode == 2u) asm volatile("griddepcontrol.launch_dependents;");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (mode != 2u) asm volatile("griddepcontrol.launch_dependents;");
+}
+
+// One launch of a fused-update kernel; p.overlap adds the programmatic-stream-serialization attribute.
+template <typename P>
+inline cudaError_t launch_update_kernel(void (*kernel)(P), dim3 grid, size_t smem, cudaStream_t stream, const UpdateParams& p) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = p.overlap ? 1u : 0u;
+    UpdateParams q = p;
+    if (q.overlap && (uint64_t)grid.x * grid.y >= 1024u) q.overlap = 2u;     // several waves: release the successor first
+    return cudaLaunchKernelEx(&cfg, kernel, q);
+}
+
 // Per-lane threshold set-up for the row with global index `grow` (row of the [B_global*H*P, N] view).
 template <int FMT, int RULE, int LPR>
 struct LaneThreshold {
@@ -177,12 +224,13 @@ struct LaneThreshold {
 
 template <int FMT, int RULE, int LPR, bool APS>
 __global__ void __launch_bounds__(kThreads) ssd_update_kernel(const UpdateParams p) {
+    grid_dependency_gate(p.overlap);
     constexpr int EPL = Fmt<FMT>::kEpl;
     constexpr int N = LPR * EPL;
     constexpr int UNR = Unroll<FMT>::value;
     constexpr unsigned FULL = 0xFFFFFFFFu;
 
-    const uint32_t step_t = p.step_t + (p.step_base ? __ldg(p.step_base) : 0u);
+    const uint32_t step_t = p.step_t + (p.step_base ? __ldcg(p.step_base) : 0u);
     const uint32_t tid = threadIdx.x;
     const uint32_t lis = tid % LPR;                 // lane in slot
     const uint32_t slot = tid / LPR;
@@ -388,6 +436,7 @@ __device__ __forceinline__ float reduce2_over_slot(float d0, float d1, uint32_t 
 // EXTRAS: any of dt_bias, in-kernel softplus, B/C groups or the z gate is in use (the plain step pays nothing for them).
 template <int FMT, int RULE, int LPR, int RPS, bool EXTRAS>
 __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateParams p) {
+    grid_dependency_gate(p.overlap);
     constexpr int EPL = Fmt<FMT>::kEpl;
     constexpr int N = LPR * EPL;
     constexpr int NSLOT = kThreads / LPR;
@@ -395,7 +444,7 @@ __global__ void __launch_bounds__(kThreads) ssd_update_tile_kernel(const UpdateP
     constexpr int GRP = RPS >= 4 ? 4 : 2;        // rows per reduction group
     static_assert(RPS % GRP == 0 && LPR >= GRP, "rows are processed GRP at a time by slots of at least GRP lanes");
 
-    const uint32_t step_t = p.step_t + (p.step_base ? __ldg(p.step_base) : 0u);
+    const uint32_t step_t = p.step_t + (p.step_base ? __ldcg(p.step_base) : 0u);
     const uint32_t lis = threadIdx.x % LPR;
     const uint32_t slot = threadIdx.x / LPR;
     const uint32_t h = blockIdx.x;                  // grid = (H, B): no index division
@@ -583,9 +632,8 @@ inline cudaError_t launch_update_one(const UpdateParams& p, cudaStream_t stream)
             if (q.P == nslot * (R)) {                                                                              \
                 note_kernel(1);                                                                                    \
                 if (q.prepare_only) return cudaSuccess;                                                            \
-                if (extras) ssd_update_tile_kernel<FMT, RULE, LPR, R, true><<<tile_grid, kThreads, 0, stream>>>(q);  \
-                else ssd_update_tile_kernel<FMT, RULE, LPR, R, false><<<tile_grid, kThreads, 0, stream>>>(q);       \
-                return cudaGetLastError();                                                                         \
+                if (extras) return launch_update_kernel(ssd_update_tile_kernel<FMT, RULE, LPR, R, true>, tile_grid, 0, stream, q);  \
+                return launch_update_kernel(ssd_update_tile_kernel<FMT, RULE, LPR, R, false>, tile_grid, 0, stream, q);             \
             }
             SSDQ_TILE_CASE(8u)
             SSDQ_TILE_CASE(4u)
@@ -602,8 +650,7 @@ inline cudaError_t launch_update_one(const UpdateParams& p, cudaStream_t stream)
     const uint32_t grid = (q.n_items + q.items_per_cta - 1) / q.items_per_cta;
     note_kernel(0);
     if (q.prepare_only) return cudaSuccess;
-    ssd_update_kernel<FMT, RULE, LPR, APS><<<grid, kThreads, 0, stream>>>(q);
-    return cudaGetLastError();
+    return launch_update_kernel(ssd_update_kernel<FMT, RULE, LPR, APS>, dim3(grid), 0, stream, q);
 }
 
 template <int FMT, int RULE, bool APS>

@@ -20,7 +20,8 @@ LIB_PATH = os.path.join(_HERE, "libssdq.so")
 EXPORTS = ("weyl_offsets_init", "ssdq_thresholds_materialize", "ssd_state_update", "quantize_store",
            "ssdq_dequantize", "ssd_decode_run", "ssd_decode_run_host", "ssd_replay_step", "ssd_decode_run_checkpointed",
            "ssd_decode_graph_create", "ssd_decode_graph_launch", "ssd_decode_graph_destroy", "ssdq_state_error_workspace_bytes", "ssdq_state_error",
-           "ssdq_state_error_static", "ssdq_readout_kl", "ssdq_copy", "ssdq_debug_status", "ssdq_last_kernel", "ssdq_last_error", "ssdq_launch_count")
+           "ssdq_state_error_static", "ssdq_readout_kl", "ssdq_copy", "ssdq_debug_status", "ssdq_last_kernel", "ssdq_last_error", "ssdq_launch_count",
+           "ssdq_set_launch_overlap")
 
 _u32, _u64, _i32, _vp = ctypes.c_uint32, ctypes.c_uint64, ctypes.c_int32, ctypes.c_void_p
 
@@ -114,6 +115,8 @@ def _load(path) -> ctypes.CDLL:
         L.ssdq_last_error.argtypes = []
         L.ssdq_launch_count.restype = _u64
         L.ssdq_launch_count.argtypes = []
+        L.ssdq_set_launch_overlap.restype = ctypes.c_int
+        L.ssdq_set_launch_overlap.argtypes = [ctypes.c_int]
         L.ssdq_debug_status.restype = ctypes.c_int
         L.ssdq_debug_status.argtypes = [ctypes.POINTER(_u32 * 4), ctypes.c_int]
     return L
@@ -343,3 +346,8 @@ def last_kernel() -> str:
 
 def launch_count() -> int:
     return int(lib().ssdq_launch_count())
+
+
+def set_launch_overlap(enabled: bool) -> bool:
+    """Programmatic dependent launch between the drivers' own kernels (on by default); returns the previous setting."""
+    return bool(lib().ssdq_set_launch_overlap(int(bool(enabled))))

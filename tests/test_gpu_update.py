@@ -645,3 +645,69 @@ def test_checkpointed_rounding_on_a_head_shard(fmt, rule):
     if sc_w is not None:
         assert torch.equal(sc_p.reshape(cfg.batch, h1 - h0, -1), sc_w.reshape(cfg.batch, cfg.nheads, -1)[:, h0:h1])
     assert torch.equal(y_p, y_w[:, :, :, h0:h1])
+
+
+@pytest.mark.parametrize("fmt,shape,sb", [(ssdq.BF16, (2, 8, 64, 128), 0), (ssdq.E4M3, (2, 8, 64, 128), 128),
+                                           (ssdq.INT8, (2, 8, 64, 128), 64 * 128), (ssdq.BF16, (3, 256, 1, 16), 0),
+                                           (ssdq.FP16, (2, 3, 8, 32), 0)])
+def test_launch_overlap_does_not_change_a_bit(fmt, shape, sb):
+    """The drivers launch their kernels with programmatic dependent launch by default (a kernel is scheduled while the one
+    before it drains and waits for it before touching memory).  Three layers, 24 steps through ssd_decode_run and through
+    a replayed graph, with the setting on and off: the same codes, scales and y, and the oracle's codes after the run."""
+    B, H, P, N = shape
+    f32 = np.float32
+    L, T = 3, 24
+    rng = np.random.default_rng(5 + fmt)
+    aps = (P == 1)
+    A = [(-np.exp(rng.uniform(-3, 1, (H, N) if aps else H))).astype(f32) for _ in range(L)]
+    D = [rng.normal(0, 0.1, H).astype(f32) for _ in range(L)]
+    xs_h = rng.standard_normal((T, L, B, H, P)).astype(f32)
+    dts_h = np.log1p(np.exp(rng.normal(-2, 0.5, (T, L, B, H)))).astype(f32)
+    Bs_h = (rng.standard_normal((T, L, B, N)) / np.sqrt(N)).astype(f32)
+    Cs_h = rng.standard_normal((T, L, B, N)).astype(f32)
+    xs, dts, Bs, Cs = (to_dev(a) for a in (xs_h, dts_h, Bs_h, Cs_h))
+
+    def fresh():
+        out = []
+        for l in range(L):
+            st_h, sc_h = oracle.new_state(shape, fmt, sb)
+            st, sc = codes_to_dev(st_h, fmt), to_dev(sc_h)
+            out.append((st, sc, ssdq.make_desc(st, sc, fmt, A=to_dev(A[l]), D=to_dev(D[l]), rule=ssdq.WEYL,
+                                               weyl=ssdq.weyl_offsets_init(l, 0, 16), layer=l, scale_block=sb)))
+        return out
+
+    def run(overlap, graph):
+        prev = ssdq.set_launch_overlap(overlap)
+        try:
+            layers = fresh()
+            y = torch.zeros_like(xs)
+            sin = ssdq.make_step_inputs(xs, dts, Bs, Cs, y)
+            descs = [d for _, _, d in layers]
+            if graph:
+                counter = torch.zeros(1, dtype=torch.int32, device="cuda")
+                g = ssdq.DecodeGraph(descs, T // 2, ssdq.make_step_inputs(xs[:T // 2], dts[:T // 2], Bs[:T // 2], Cs[:T // 2], y[:T // 2]), counter)
+                g.launch()
+                g.launch()
+                torch.cuda.synchronize()
+                g.close()
+            else:
+                ssdq.ssd_decode_run(descs, 1, T, sin)
+                torch.cuda.synchronize()
+            return layers, y
+        finally:
+            ssdq.set_launch_overlap(prev)
+
+    assert ssdq.set_launch_overlap(True) is True           # on by default
+    base = None
+    for graph in (True, False):         # the graph replays the first half of the inputs twice: compared with itself only
+        base, y0 = run(False, graph)
+        got, y = run(True, graph)
+        for (s0, c0, _), (s1, c1, _) in zip(base, got):
+            assert torch.equal(s0, s1) and (c0 is None or torch.equal(c0, c1)), graph
+        assert torch.equal(y0, y), graph
+    # and the run is the oracle's (first layer)
+    st_h, sc_h = oracle.new_state(shape, fmt, sb)
+    for t in range(1, T + 1):
+        oracle.state_update(st_h, sc_h, fmt, sb, xs_h[t - 1, 0], dts_h[t - 1, 0], A[0], Bs_h[t - 1, 0], Cs_h[t - 1, 0], D[0],
+                            oracle.WEYL, t, layer=0, weyl_block=16)
+    assert np.array_equal(codes_to_host(base[0][0], fmt), st_h)
