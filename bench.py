@@ -34,8 +34,8 @@ FALLBACK_HBM_GBS = 6650.0      # an earlier stream-copy measurement on this machine
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the fused update kernel from the one-kernel ncu
 # captures summarised under profiles/ (same kernel and per-layer shape as the benchmark's launches; see NCU_TRAFFIC_SOURCE).
 # A launch ends with part of its last writes still in L2, so the write term undercounts by up to the L2 size.
-NCU_TRAFFIC_BYTES = {(5, "weyl"): 272_967_936 + 215_749_376, (5, "rtn"): 272_995_072 + 215_929_088,
-                     (3, "weyl"): 85_321_216 + 26_518_272, (3, "rtn"): 85_298_176 + 28_177_408,
+NCU_TRAFFIC_BYTES = {(5, "weyl"): 272_957_184 + 216_289_792, (5, "rtn"): 272_980_224 + 216_325_376,
+                     (3, "weyl"): 85_328_896 + 27_483_392, (3, "rtn"): 85_310_208 + 28_491_520,
                      (4, "weyl"): 17_901_056 + 0, (4, "rtn"): 17_884_672 + 0}
 NCU_TRAFFIC_SOURCE = {5: "profiles/ssd_update_tile_kernel_bf16_config5.md (one launch, 2 layers resident; ~57 MB of the writes still in L2 at launch end)",
                       3: "profiles/ssd_update_tile_kernel_fp16_config3.md (state smaller than L2: writes mostly stay there)",

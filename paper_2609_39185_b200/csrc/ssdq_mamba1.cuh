@@ -7,6 +7,8 @@
 // issued two entries at a time with the packed binary32 instructions.  Consecutive lanes own consecutive channels, so
 // the state, dt, x and y accesses of a warp are contiguous.
 #pragma once
+#include <cstddef>
+#include <type_traits>
 #include "ssdq_update.cuh"
 
 namespace ssdq {
@@ -49,6 +51,24 @@ __device__ __forceinline__ f32x2 exp_spec2(f32x2 z2) {
 // by its first eight lanes.  Channels beyond H (last tile only) run on a clamped channel and store nothing.
 // With the loads out of the way the kernel is bound by instruction issue (every entry needs its own exponential), so
 // the dithered rules, which need more registers, trade two resident CTAs for a spill-free loop (measured).
+// The loop is unrolled over the two stages so that every shared-memory address is a per-thread base plus a constant,
+// and rows are addressed by a 32-bit index (B * H < 2^32) widened once per access: the ring costs ~25 instructions per row.
+template <int SOFF, int GOFF>
+__device__ __forceinline__ void cp_async16_ca_at(uint32_t smem_base, const void* gmem_base) {
+    asm volatile("cp.async.ca.shared.global [%0 + %2], [%1 + %3], 16;" ::"r"(smem_base), "l"(gmem_base), "n"(SOFF), "n"(GOFF) : "memory");
+}
+template <int SOFF>
+__device__ __forceinline__ void cp_async4_ca_at(uint32_t smem_base, const void* gmem) {
+    asm volatile("cp.async.ca.shared.global [%0 + %2], [%1], 4;" ::"r"(smem_base), "l"(gmem), "n"(SOFF) : "memory");
+}
+
+template <int CH>
+struct Mamba1Stage {
+    uint4 codes[CH][kThreads];
+    float bc[kThreads / 32][32];        // per warp: B[0..15], C[0..15] of the sequence
+    float dt[kThreads], x[kThreads], sc[kThreads];
+};
+
 template <int FMT, int RULE>
 __global__ void __launch_bounds__(kThreads, RULE == RULE_RTN ? 8 : 6) ssd_update_mamba1_kernel(const UpdateParams p) {
     grid_dependency_gate(p.overlap);
@@ -56,9 +76,8 @@ __global__ void __launch_bounds__(kThreads, RULE == RULE_RTN ? 8 : 6) ssd_update
     constexpr int N = 16;
     constexpr int CH = N / EPL;                         // chunks per row: 2 or 1
     constexpr unsigned FULL = 0xFFFFFFFFu;
-    __shared__ __align__(16) uint4 s_codes[2][CH][kThreads];
-    __shared__ __align__(16) float s_bc[2][kThreads / 32][2 * N];     // per warp: B[0..15], C[0..15] of the sequence
-    __shared__ float s_dt[2][kThreads], s_x[2][kThreads], s_sc[2][kThreads];
+    using Stage = Mamba1Stage<CH>;
+    __shared__ __align__(16) Stage ring[2];
 
     const uint32_t step_t = p.step_t + (p.step_base ? __ldcg(p.step_base) : 0u);
     const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
@@ -85,54 +104,59 @@ __global__ void __launch_bounds__(kThreads, RULE == RULE_RTN ? 8 : 6) ssd_update
     // Weyl: a row is one dither block (block 16 = N): r = global row, c = n
     const uint32_t weyl_const = p.weyl.mul_row + p.weyl.mul_col + p.weyl.base + step_t * p.weyl.phi;
 
-    const uint32_t codes_s = (uint32_t)__cvta_generic_to_shared(&s_codes[0][0][tid]);     // + stage * CH * kThreads * 16 + c * kThreads * 16
-    const uint32_t dt_s = (uint32_t)__cvta_generic_to_shared(&s_dt[0][tid]);              // + stage * kThreads * 4
-    const uint32_t x_s = (uint32_t)__cvta_generic_to_shared(&s_x[0][tid]);
-    const uint32_t sc_s = (uint32_t)__cvta_generic_to_shared(&s_sc[0][tid]);
-    const uint32_t bc_s = (uint32_t)__cvta_generic_to_shared(&s_bc[0][warp][(lane & 7u) * 4u]);   // + stage * sizeof(s_bc[0])
-    uint32_t ok_bits = 0;                               // bit s: the row in stage s passed the debug build's range checks
-    auto issue = [&](uint32_t b, uint32_t stage) {
-        const uint64_t row = (uint64_t)b * p.H + d;
-        // debug builds: the row's vectors, its x / y / dt elements, its scale and the sequence's B and C
-        bool ok = SSDQ_RANGE_OK(p, DBG_STATE, row * CH, CH, state_vecs) && SSDQ_RANGE_OK(p, DBG_ROWS, row, 1, rows) &&
+    const uint32_t ring_s = (uint32_t)__cvta_generic_to_shared(&ring[0]);
+    const uint32_t t16 = ring_s + tid * 16u, t4 = ring_s + tid * 4u;                 // this thread's 16-byte and 4-byte cells
+    const uint32_t bcw = ring_s + warp * 128u + (lane & 7u) * 16u;                   // lanes 0-7: one 16-byte chunk of the warp's B | C
+    const float* bc_src = (lane < 4u ? p.Bm : p.Cm) + (lane & 3u) * 4u;
+    const char* state_c = reinterpret_cast<const char*>(p.state);
+    char* state_w = reinterpret_cast<char*>(p.state);
+#ifdef SSDQ_DEBUG
+    uint32_t ok_bits = 0;                               // bit s: the row in stage s passed the range checks
+#endif
+
+    auto issue = [&](uint32_t b, auto stage_c) {
+        constexpr int S = decltype(stage_c)::value;
+        constexpr int SO = S * (int)sizeof(Stage);
+        const uint32_t row = b * p.H + d;
+#ifdef SSDQ_DEBUG
+        // the row's vectors, its x / y / dt elements, its scale and the sequence's B and C
+        bool ok = SSDQ_RANGE_OK(p, DBG_STATE, (uint64_t)row * CH, CH, state_vecs) && SSDQ_RANGE_OK(p, DBG_ROWS, row, 1, rows) &&
                   SSDQ_RANGE_OK(p, DBG_ITEMS, row, 1, items) && SSDQ_RANGE_OK(p, DBG_BC, (size_t)b * N, N, bc_floats);
         if constexpr (Fmt<FMT>::kScaled) ok = ok && SSDQ_RANGE_OK(p, DBG_SCALES, row, 1, scales);
-#ifdef SSDQ_DEBUG
-        ok = __all_sync(FULL, ok);                      // lanes copy one another's rows and meet at warp barriers: skip as a warp
-#endif
-        ok_bits = (ok_bits & ~(1u << stage)) | ((uint32_t)ok << stage);
+        ok = __all_sync(FULL, ok);                      // lanes meet at warp barriers and share B / C: skip as a warp
+        ok_bits = (ok_bits & ~(1u << S)) | ((uint32_t)ok << S);
         if (!ok) return;
+#endif
         // .ca: a two-byte row is two 16-byte chunks 32 bytes apart per lane, so each copy instruction touches every
         // sector of the warp's kilobyte; keeping the lines in L1 lets the second one hit there
-        const uint4* sp = reinterpret_cast<const uint4*>(p.state) + row * CH;
-#pragma unroll
-        for (int c = 0; c < CH; ++c) cp_async16_ca(codes_s + (stage * CH + c) * (kThreads * 16u), sp + c);
-        cp_async4_ca(dt_s + stage * (kThreads * 4u), p.dt + row);
-        cp_async4_ca(x_s + stage * (kThreads * 4u), p.x + row);
-        if constexpr (Fmt<FMT>::kScaled) cp_async4_ca(sc_s + stage * (kThreads * 4u), p.scales + row);
-        if (lane < 8u) cp_async16_ca(bc_s + stage * (uint32_t)sizeof(s_bc[0]), (lane < 4u ? p.Bm : p.Cm) + (size_t)b * N + (lane & 3u) * 4u);
+        const char* sp = state_c + (uint64_t)row * (CH * 16u);
+        cp_async16_ca_at<SO + (int)offsetof(Stage, codes), 0>(t16, sp);
+        if constexpr (CH == 2) cp_async16_ca_at<SO + (int)offsetof(Stage, codes) + kThreads * 16, 16>(t16, sp);
+        cp_async4_ca_at<SO + (int)offsetof(Stage, dt)>(t4, p.dt + row);
+        cp_async4_ca_at<SO + (int)offsetof(Stage, x)>(t4, p.x + row);
+        if constexpr (Fmt<FMT>::kScaled) cp_async4_ca_at<SO + (int)offsetof(Stage, sc)>(t4, p.scales + row);
+        if (lane < 8u) cp_async16_ca_at<SO + (int)offsetof(Stage, bc), 0>(bcw, bc_src + (size_t)b * N);
     };
-    issue(b_first, 0u);
-    cp_async_commit();
 
-    uint32_t stage = 0;
-    for (uint32_t b = b_first; b < b_last; ++b, stage ^= 1u) {
+    auto row_step = [&](uint32_t b, auto stage_c) {
+        constexpr int S = decltype(stage_c)::value;
         __syncwarp(FULL);                               // every lane is done with the B / C of the stage refilled next
-        if (b + 1 < b_last) issue(b + 1, stage ^ 1u);
+        if (b + 1 < b_last) issue(b + 1, std::integral_constant<int, 1 - S>{});
         cp_async_commit();
         cp_async_wait<1>();                             // this row's group has landed (the next one may be pending)
         __syncwarp(FULL);                               // ... also the B / C chunks that other lanes copied
-        if (!((ok_bits >> stage) & 1u)) continue;                 // debug builds only, and then the whole warp
-        const uint64_t row = (uint64_t)b * p.H + d;
-        const uint64_t grow = row + p.row_off0 + (uint64_t)b * p.row_skip;
-        uint4* sp = reinterpret_cast<uint4*>(p.state) + row * CH;
+#ifdef SSDQ_DEBUG
+        if (!((ok_bits >> S) & 1u)) return;             // the whole warp
+#endif
+        const Stage& st = ring[S];
+        const uint32_t row = b * p.H + d;
         uint4 raw[CH];
 #pragma unroll
-        for (int c = 0; c < CH; ++c) raw[c] = s_codes[stage][c][tid];
-        const float dtv = s_dt[stage][tid], xv = s_x[stage][tid];
+        for (int c = 0; c < CH; ++c) raw[c] = st.codes[c][tid];
+        const float dtv = st.dt[tid], xv = st.x[tid];
         float sc_old = 0.0f;
-        if constexpr (Fmt<FMT>::kScaled) sc_old = s_sc[stage][tid];
-        const float4* Bp = reinterpret_cast<const float4*>(&s_bc[stage][warp][0]);       // the same address in every lane: a broadcast
+        if constexpr (Fmt<FMT>::kScaled) sc_old = st.sc[tid];
+        const float4* Bp = reinterpret_cast<const float4*>(&st.bc[warp][0]);            // the same address in every lane: a broadcast
         const float4* Cp = Bp + N / 4;
         const float dtx = __fmul_rn(dtv, xv);
         const f32x2 dt2 = pack2(dtv, dtv), dtx2 = pack2(dtx, dtx), sc2 = pack2(sc_old, sc_old);
@@ -180,10 +204,16 @@ __global__ void __launch_bounds__(kThreads, RULE == RULE_RTN ? 8 : 6) ssd_update
 #pragma unroll
             for (int q = 0; q < N / 2; ++q) unpack2(hn[q], v[2 * q], v[2 * q + 1]);
         }
-        const uint64_t flat0 = grow * N;
+        // global row = local row + row_off0 + b * row_skip; the Weyl accumulator needs it modulo 2^32 only
+        uint64_t flat0 = 0;
         uint32_t acc_row = 0;
-        if constexpr (RULE == RULE_WEYL) acc_row = weyl_const + p.weyl.mul_row * (uint32_t)grow;
-        if constexpr (RULE == RULE_SR_HASH) acc_row = (uint32_t)flat0 * kHashP1 + ((uint32_t)(flat0 >> 32) ^ key1) * kHashP5 + hash_base;
+        if constexpr (RULE == RULE_WEYL) {
+            acc_row = weyl_const + p.weyl.mul_row * (row + (uint32_t)p.row_off0 + b * p.row_skip);
+        } else if constexpr (RULE != RULE_RTN) {
+            flat0 = ((uint64_t)row + p.row_off0 + (uint64_t)b * p.row_skip) * N;
+            if constexpr (RULE == RULE_SR_HASH) acc_row = (uint32_t)flat0 * kHashP1 + ((uint32_t)(flat0 >> 32) ^ key1) * kHashP5 + hash_base;
+        }
+        uint4* sp = reinterpret_cast<uint4*>(state_w + (uint64_t)row * (CH * 16u));
 #pragma unroll
         for (int c = 0; c < CH; ++c) {
             const uint64_t g = (flat0 + (uint64_t)c * EPL) >> 2;
@@ -194,6 +224,13 @@ __global__ void __launch_bounds__(kThreads, RULE == RULE_RTN ? 8 : 6) ssd_update
                                                             key0, key1, p.scale_top);
             if (active) sp[c] = packed;
         }
+    };
+
+    issue(b_first, std::integral_constant<int, 0>{});
+    cp_async_commit();
+    for (uint32_t b = b_first; b < b_last; b += 2) {
+        row_step(b, std::integral_constant<int, 0>{});
+        if (b + 1 < b_last) row_step(b + 1, std::integral_constant<int, 1>{});
     }
     cp_async_wait<0>();
 }

@@ -649,7 +649,8 @@ def test_checkpointed_rounding_on_a_head_shard(fmt, rule):
 
 @pytest.mark.parametrize("fmt,shape,sb", [(ssdq.BF16, (2, 8, 64, 128), 0), (ssdq.E4M3, (2, 8, 64, 128), 128),
                                            (ssdq.INT8, (2, 8, 64, 128), 64 * 128), (ssdq.BF16, (3, 256, 1, 16), 0),
-                                           (ssdq.FP16, (2, 3, 8, 32), 0)])
+                                           (ssdq.FP16, (2, 3, 8, 32), 0),
+                                           (ssdq.BF16, (16, 64, 64, 128), 0)])      # 1024 CTAs: the many-wave order of the gate
 def test_launch_overlap_does_not_change_a_bit(fmt, shape, sb):
     """The drivers launch their kernels with programmatic dependent launch by default (a kernel is scheduled while the one
     before it drains and waits for it before touching memory).  Three layers, 24 steps through ssd_decode_run and through

@@ -65,3 +65,11 @@ def test_two_replicas_equal_one_big_batch(tmp_path):
         assert np.array_equal(np.concatenate([p[name] for p in parts]), full)
         assert np.array_equal(np.concatenate([p[name + "_heads"] for p in parts], axis=1), full)
         assert all(float(p["slowest"]) == 2.0 for p in parts)
+
+
+def test_head_ranges_tile_the_layer():
+    import pytest
+    from paper_2609_39185_b200.replicas import shard_head_range
+    assert [shard_head_range(r, 4, 128) for r in range(4)] == [(0, 32), (32, 64), (64, 96), (96, 128)]
+    with pytest.raises(ValueError):
+        shard_head_range(0, 3, 128)
