@@ -16,8 +16,11 @@
 #pragma once
 #include "ssdq_update.cuh"
 
+#ifndef SSDQ_STREAM_STAGES
+#define SSDQ_STREAM_STAGES 2
+#endif
 #ifndef SSDQ_STREAM_MINB
-#define SSDQ_STREAM_MINB 5
+#define SSDQ_STREAM_MINB 4
 #endif
 
 namespace ssdq {
@@ -297,7 +300,7 @@ inline cudaError_t launch_stream(const UpdateParams& p, cudaStream_t stream) {
 
 // Shapes covered: N = 128 with heads of 64 or 128 rows, the plain signature (no dt_bias / softplus / groups / gate),
 // x, y and the scales 16-byte aligned.  Two stages: one item in flight per CTA besides the one being computed was
-// the fastest setting measured (more stages cost resident CTAs).
+// the fastest setting measured (a third stage was slower at every occupancy tried).
 template <int FMT, int RULE, int LPR>
 cudaError_t try_launch_stream(const UpdateParams& p, cudaStream_t stream, bool& launched) {
     launched = false;
@@ -309,8 +312,8 @@ cudaError_t try_launch_stream(const UpdateParams& p, cudaStream_t stream, bool& 
         launched = true;
         const bool row_scale = p.scale_block == (uint32_t)(LPR * 16);
         if (p.P == nslot * 4u)
-            return row_scale ? launch_stream<FMT, RULE, LPR, 4, 2, true>(p, stream) : launch_stream<FMT, RULE, LPR, 4, 2, false>(p, stream);
-        return row_scale ? launch_stream<FMT, RULE, LPR, 8, 2, true>(p, stream) : launch_stream<FMT, RULE, LPR, 8, 2, false>(p, stream);
+            return row_scale ? launch_stream<FMT, RULE, LPR, 4, SSDQ_STREAM_STAGES, true>(p, stream) : launch_stream<FMT, RULE, LPR, 4, SSDQ_STREAM_STAGES, false>(p, stream);
+        return row_scale ? launch_stream<FMT, RULE, LPR, 8, SSDQ_STREAM_STAGES, true>(p, stream) : launch_stream<FMT, RULE, LPR, 8, SSDQ_STREAM_STAGES, false>(p, stream);
     }
     return cudaSuccess;
 }
