@@ -75,6 +75,8 @@ def lib() -> ctypes.CDLL:
                                           i32, u32, u32, u32, u64, u32, u32, vp, i32, u32, vp, u32, u32]
         L.oracle_softplus_spec.restype = f32
         L.oracle_softplus_spec.argtypes = [f32]
+        L.oracle_softplus_spec_array.restype = None
+        L.oracle_softplus_spec_array.argtypes = [vp, u64, vp]
         L.oracle_quantize_store.restype = i32
         L.oracle_quantize_store.argtypes = [vp, vp, vp, u64, u32, i32, u32, i32, u32, u32, u32, u64, u64, u32]
         L.oracle_replay_step.restype = i32
@@ -173,7 +175,9 @@ def decode(codes, fmt):
 # ---- the decode step ------------------------------------------------------------------------
 def softplus_spec(x):
     x = _f32(np.atleast_1d(x))
-    return np.array([lib().oracle_softplus_spec(float(v)) for v in x.ravel()], dtype=np.float32).reshape(x.shape)
+    out = np.empty_like(x)
+    lib().oracle_softplus_spec_array(_ptr(x), x.size, _ptr(out))
+    return out
 
 
 def state_update(state, scales, fmt, scale_block, x, dt, A, Bm, Cm, D, rule, step_t, *, layer=0,

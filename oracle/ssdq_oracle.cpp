@@ -325,6 +325,10 @@ void oracle_philox4x32_10(const uint32_t* ctr, const uint32_t* key, uint32_t* ou
 float oracle_exp_spec(float z) { return exp_spec(z); }
 uint32_t oracle_fmix32(uint32_t h) { return fmix32(h); }
 float oracle_softplus_spec(float x) { return softplus_spec(x); }
+void oracle_softplus_spec_array(const float* x, uint64_t n, float* out) {
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < (int64_t)n; ++i) out[i] = softplus_spec(x[i]);
+}
 float oracle_round(float v, int fmt, int rule, uint32_t U) { return round_on_grid(v, fmt, rule, U); }
 uint32_t oracle_encode(float q, int fmt) { return encode(q, fmt); }
 float oracle_decode(uint32_t code, int fmt) { return decode(code, fmt); }
@@ -347,7 +351,8 @@ void oracle_round_encode_array(const float* v, const uint32_t* U, uint64_t n_U, 
     }
 }
 void oracle_exp_spec_array(const float* z, uint64_t n, float* out) {
-    for (uint64_t i = 0; i < n; ++i) out[i] = exp_spec(z[i]);
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < (int64_t)n; ++i) out[i] = exp_spec(z[i]);
 }
 
 // ---- one decode step of one layer (Eq. 1 + readout + Eq. 2), in place -----------------------

@@ -10,6 +10,9 @@ column multipliers are zero gives every entry the accumulator `base`) and the re
 BF16, FP16: all 2^32 - 2^24 finite patterns.  E4M3, INT8: all patterns with |v| <= 448 (127), each block of 16 entries
 led by the format's top value so that its scale is exactly 1 and the value reaches the rounding unchanged (what lies
 beyond the top cannot occur after scaling).  NaN and infinity are outside the precondition (finite inputs).
+
+The fixed binary32 routines of Eq. 1 -- the exponential in its scalar and its packed form, and the softplus of the
+in-kernel step size -- are compared the same way, on every finite argument, through the fused step itself.
 """
 import numpy as np
 import pytest
@@ -105,3 +108,87 @@ def test_every_binary32_in_range_through_the_one_byte_stores(fmt, top, mode):
             assert np.all(scales.cpu().numpy() == 1.0)
             assert np.all(got[:, 0] == top_code)                          # the pinning entry itself: floor(top + u) = top
             assert _first_mismatch(got[:, 1:], want[:, 1:], src[:, 1:]) is None, (sign, c, _first_mismatch(got[:, 1:], want[:, 1:], src[:, 1:]))
+
+
+def _finite_chunks(chunk):
+    """All finite binary32 patterns, `chunk` at a time (NaN and infinity, exponent field 255, replaced by 0)."""
+    lane = np.arange(chunk, dtype=np.uint32)
+    for c in range((1 << 32) // chunk):
+        bits = lane + np.uint32(c * chunk)
+        if ((c * chunk) >> 23) & 0xFF == 0xFF or (((c + 1) * chunk - 1) >> 23) & 0xFF == 0xFF:
+            bits[(bits & 0x7F800000) == 0x7F800000] = 0
+        yield c, bits
+
+
+def test_every_binary32_argument_of_the_scalar_exponential():
+    """exp_spec (Eq. 1's decay a = exp(dt A), evaluated by the fixed binary32 routine) for EVERY finite argument: the
+    FP32 twin with one decay per state stores h' = fma(a, 1, 0) = a unrounded, so with h = 1, x = 0 and dt = 1 the state
+    after one step is exp_spec(A) entry for entry."""
+    H, N = 1 << 22, 16
+    f32 = np.float32
+    ones = torch.ones((1, H, 1, N), dtype=torch.float32, device="cuda")
+    st = torch.empty_like(ones)
+    x = torch.zeros((1, H, 1), device="cuda"); dt = torch.ones((1, H), device="cuda")
+    Bm = torch.ones((1, N), device="cuda"); Cm = torch.zeros((1, N), device="cuda"); y = torch.empty_like(x)
+    A = torch.empty((H, N), dtype=torch.float32, device="cuda")
+    desc = ssdq.make_desc(st, None, ssdq.FP32, A=A, D=None, rule=ssdq.RTN)
+    for c, bits in _finite_chunks(H * N):
+        z = bits.view(f32)
+        A.copy_(torch.from_numpy(z.reshape(H, N)))
+        st.copy_(ones)
+        ssdq.ssd_state_update(desc, 1, x=x, dt=dt, Bm=Bm, Cm=Cm, y=y)
+        assert ssdq.last_kernel() == "ssd_update_kernel"
+        want = oracle.exp_spec(z)
+        got = st.cpu().numpy().reshape(-1)
+        assert _first_mismatch(got.view(np.uint32), want.view(np.uint32), z) is None, (c, _first_mismatch(got.view(np.uint32), want.view(np.uint32), z))
+
+
+def test_every_binary32_argument_of_the_packed_exponential():
+    """The Mamba-1 kernel evaluates the same routine on packed pairs (exp_spec2).  Its state is rounded to the store, so
+    the decay is read through the readout instead: h = 1, x = 0, dt = 1 and C = the n-th unit vector give y = a[d, n]
+    exactly; sixteen launches, one per column, cover the sixteen distinct arguments of every row."""
+    H, N = 1 << 22, 16
+    f32 = np.float32
+    ones = torch.full((1, H, 1, N), 0x3F80, dtype=torch.int16, device="cuda")          # 1.0 in BF16
+    st = torch.empty_like(ones)
+    x = torch.zeros((1, H, 1), device="cuda"); dt = torch.ones((1, H), device="cuda")
+    Bm = torch.ones((1, N), device="cuda"); y = torch.empty_like(x)
+    A = torch.empty((H, N), dtype=torch.float32, device="cuda")
+    desc = ssdq.make_desc(st, None, ssdq.BF16, A=A, D=None, rule=ssdq.RTN)
+    onehot = [torch.zeros((1, N), device="cuda") for _ in range(N)]
+    for n in range(N):
+        onehot[n][0, n] = 1.0
+    got = torch.empty((H, N), dtype=torch.float32, device="cuda")
+    for c, bits in _finite_chunks(H * N):
+        z = bits.view(f32)
+        A.copy_(torch.from_numpy(z.reshape(H, N)))
+        for n in range(N):
+            st.copy_(ones)
+            ssdq.ssd_state_update(desc, 1, x=x, dt=dt, Bm=Bm, Cm=onehot[n], y=y)
+            got[:, n] = y.reshape(-1)
+        assert ssdq.last_kernel() == "ssd_update_mamba1_kernel"
+        want = oracle.exp_spec(z)
+        g = got.cpu().numpy().reshape(-1)
+        assert _first_mismatch(g.view(np.uint32), want.view(np.uint32), z) is None, (c, _first_mismatch(g.view(np.uint32), want.view(np.uint32), z))
+
+
+def test_every_binary32_argument_of_the_softplus():
+    """softplus_spec (the in-kernel step size dt <- softplus(dt + dt_bias) of a production signature, Appendix B "Runners")
+    for EVERY finite argument: with h = 0, A = 0 (a = 1), x = 1, B = 1 the update is h' = fma(1, 0, (dt' * 1) * 1) = dt',
+    and C = the first unit vector reads it out as y."""
+    H, N = 1 << 22, 16
+    f32 = np.float32
+    st = torch.zeros((1, H, 1, N), dtype=torch.float32, device="cuda")
+    x = torch.ones((1, H, 1), device="cuda"); dt = torch.empty((1, H), device="cuda")
+    Bm = torch.ones((1, N), device="cuda"); Cm = torch.zeros((1, N), device="cuda"); y = torch.empty_like(x)
+    Cm[0, 0] = 1.0
+    A = torch.zeros((H,), dtype=torch.float32, device="cuda")
+    desc = ssdq.make_desc(st, None, ssdq.FP32, A=A, D=None, rule=ssdq.RTN, dt_softplus=True)
+    for c, bits in _finite_chunks(H):
+        z = bits.view(f32)
+        dt.copy_(torch.from_numpy(z.reshape(1, H)))
+        st.zero_()
+        ssdq.ssd_state_update(desc, 1, x=x, dt=dt, Bm=Bm, Cm=Cm, y=y)
+        want = oracle.softplus_spec(z)
+        got = y.cpu().numpy().reshape(-1)
+        assert _first_mismatch(got.view(np.uint32), want.view(np.uint32), z) is None, (c, _first_mismatch(got.view(np.uint32), want.view(np.uint32), z))
