@@ -75,6 +75,8 @@ def lib() -> ctypes.CDLL:
                                           i32, u32, u32, u32, u64, u32, u32, vp, i32, u32, vp, u32, u32]
         L.oracle_softplus_spec.restype = f32
         L.oracle_softplus_spec.argtypes = [f32]
+        L.oracle_block_scale_array.restype = None
+        L.oracle_block_scale_array.argtypes = [vp, u64, i32, vp]
         L.oracle_softplus_spec_array.restype = None
         L.oracle_softplus_spec_array.argtypes = [vp, u64, vp]
         L.oracle_quantize_store.restype = i32
@@ -177,6 +179,14 @@ def softplus_spec(x):
     x = _f32(np.atleast_1d(x))
     out = np.empty_like(x)
     lib().oracle_softplus_spec_array(_ptr(x), x.size, _ptr(out))
+    return out
+
+
+def block_scale(amax, fmt):
+    """FP32 block scale max(amax / top, FLT_MIN) of a scaled store (top = 448 for E4M3, q_max for INTb), elementwise."""
+    amax = _f32(np.atleast_1d(amax))
+    out = np.empty_like(amax)
+    lib().oracle_block_scale_array(_ptr(amax), amax.size, fmt, _ptr(out))
     return out
 
 

@@ -325,6 +325,11 @@ void oracle_philox4x32_10(const uint32_t* ctr, const uint32_t* key, uint32_t* ou
 float oracle_exp_spec(float z) { return exp_spec(z); }
 uint32_t oracle_fmix32(uint32_t h) { return fmix32(h); }
 float oracle_softplus_spec(float x) { return softplus_spec(x); }
+// the block scale of a scaled store for an array of block maxima (exported so that it can be pinned on its own)
+void oracle_block_scale_array(const float* amax, uint64_t n, int fmt, float* out) {
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < (int64_t)n; ++i) out[i] = block_scale(amax[i], fmt);
+}
 void oracle_softplus_spec_array(const float* x, uint64_t n, float* out) {
 #pragma omp parallel for schedule(static)
     for (int64_t i = 0; i < (int64_t)n; ++i) out[i] = softplus_spec(x[i]);

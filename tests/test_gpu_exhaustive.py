@@ -192,3 +192,30 @@ def test_every_binary32_argument_of_the_softplus():
         want = oracle.softplus_spec(z)
         got = y.cpu().numpy().reshape(-1)
         assert _first_mismatch(got.view(np.uint32), want.view(np.uint32), z) is None, (c, _first_mismatch(got.view(np.uint32), want.view(np.uint32), z))
+
+
+@pytest.mark.parametrize("fmt", [ssdq.E4M3, ssdq.INT8, ssdq.INT7, ssdq.INT6, ssdq.INT4])
+def test_every_positive_binary32_maximum_through_the_scale_of_the_persistent_kernel(fmt):
+    """The persistent one-byte kernel divides the row maximum by the format's constant with a multiply and two fused
+    corrections instead of a division.  Every positive finite binary32 maximum: with h = 0, A = 0, dt = 1 and B the first
+    unit vector a row's only non-zero entry is h' = x, so its maximum is x and its stored scale must be the oracle's
+    max(x / top, FLT_MIN), bit for bit."""
+    B, H, P, N = 128, 128, 64, 128
+    rows = B * H * P
+    st = torch.zeros((B, H, P, N), dtype=torch.uint8, device="cuda")
+    sc = torch.ones((rows,), dtype=torch.float32, device="cuda")
+    x = torch.empty((B, H, P), device="cuda"); dt = torch.ones((B, H), device="cuda"); y = torch.empty_like(x)
+    Bm = torch.zeros((B, N), device="cuda"); Bm[:, 0] = 1.0
+    Cm = torch.zeros((B, N), device="cuda")
+    A = torch.zeros((H,), device="cuda")
+    desc = ssdq.make_desc(st, sc, fmt, A=A, D=None, rule=ssdq.RTN, scale_block=N)
+    lane = np.arange(rows, dtype=np.uint32)
+    for c in range(0x7F800000 // rows):
+        amax = (lane + np.uint32(c * rows)).view(np.float32)
+        x.copy_(torch.from_numpy(amax.reshape(B, H, P)))
+        st.zero_()
+        ssdq.ssd_state_update(desc, 1, x=x, dt=dt, Bm=Bm, Cm=Cm, y=y)
+        assert ssdq.last_kernel() == "ssd_update_stream_kernel"
+        want = oracle.block_scale(amax, fmt)
+        got = sc.cpu().numpy()
+        assert _first_mismatch(got.view(np.uint32), want.view(np.uint32), amax) is None, (c, _first_mismatch(got.view(np.uint32), want.view(np.uint32), amax))

@@ -227,3 +227,18 @@ def test_head_scale_absorbs_a_shared_decay():
                             None, RTN, t, weyl_block=128)
     assert np.array_equal(state, before)
     assert np.allclose(scales / s_before, np.exp(0.1 * A.astype(np.float64)) ** 19, rtol=1e-5)
+
+
+def test_block_scale_is_the_ieee_quotient_floored_at_the_smallest_normal():
+    """s = max|h'| / top in FP32 (Appendix B "Formats"): against the quotient taken in double and rounded once (a double
+    quotient of two binary32 numbers rounds to the binary32 quotient: 53 >= 2 * 24 + 2), for random maxima, powers of
+    two, subnormals and zero, each format's top."""
+    rng = np.random.default_rng(3)
+    amax = np.concatenate([np.abs(rng.standard_normal(4000)).astype(np.float32) * np.float32(10.0) ** rng.integers(-38, 38, 4000).astype(np.float32),
+                           np.float32(2.0) ** np.arange(-149, 128, dtype=np.float32), np.zeros(1, np.float32),
+                           rng.integers(1, 1 << 23, 500).astype(np.uint32).view(np.float32)])
+    amax = amax[np.isfinite(amax)]
+    tiny = np.float32(np.finfo(np.float32).tiny)
+    for fmt, top in ((oracle.E4M3, 448.0), (oracle.INT8, 127.0), (oracle.INT7, 63.0), (oracle.INT6, 31.0), (oracle.INT4, 7.0)):
+        want = np.maximum((amax.astype(np.float64) / top).astype(np.float32), tiny)
+        assert np.array_equal(oracle.block_scale(amax, fmt), want)
