@@ -651,13 +651,14 @@ def test_checkpointed_rounding_on_a_head_shard(fmt, rule):
                                            (ssdq.INT8, (2, 8, 64, 128), 64 * 128), (ssdq.BF16, (3, 256, 1, 16), 0),
                                            (ssdq.FP16, (2, 3, 8, 32), 0),
                                            (ssdq.BF16, (16, 64, 64, 128), 0)])      # 1024 CTAs: the many-wave order of the gate
-def test_launch_overlap_does_not_change_a_bit(fmt, shape, sb):
+@pytest.mark.parametrize("L", [1, 3])       # one layer: every launch reads what the launch just before it wrote
+def test_launch_overlap_does_not_change_a_bit(fmt, shape, sb, L):
     """The drivers launch their kernels with programmatic dependent launch by default (a kernel is scheduled while the one
     before it drains and waits for it before touching memory).  Three layers, 24 steps through ssd_decode_run and through
     a replayed graph, with the setting on and off: the same codes, scales and y, and the oracle's codes after the run."""
     B, H, P, N = shape
     f32 = np.float32
-    L, T = 3, 24
+    T = 24 if L == 3 else 48
     rng = np.random.default_rng(5 + fmt)
     aps = (P == 1)
     A = [(-np.exp(rng.uniform(-3, 1, (H, N) if aps else H))).astype(f32) for _ in range(L)]
@@ -712,3 +713,41 @@ def test_launch_overlap_does_not_change_a_bit(fmt, shape, sb):
         oracle.state_update(st_h, sc_h, fmt, sb, xs_h[t - 1, 0], dts_h[t - 1, 0], A[0], Bs_h[t - 1, 0], Cs_h[t - 1, 0], D[0],
                             oracle.WEYL, t, layer=0, weyl_block=16)
     assert np.array_equal(codes_to_host(base[0][0], fmt), st_h)
+
+
+@pytest.mark.parametrize("cfg_index,batch,fmt", [(4, 0, None), (5, 32, None), (5, 32, ssdq.INT8), (2, 512, None), (3, 0, None)])
+def test_launch_overlap_at_full_size_on_one_layer(cfg_index, batch, fmt):
+    """Full-size launches of one layer back to back (every kernel reads the state, and for the scaled stores the scales,
+    that the kernel just before it wrote, on whichever SM it lands): 16 steps through ssd_decode_run with the
+    programmatic-launch setting on and off end in the same codes, scales and y."""
+    from dataclasses import replace
+    cfg = replace(workloads.CONFIGS[cfg_index], n_layers=1)
+    if batch:
+        cfg = cfg.with_batch(batch)
+    if fmt is not None:
+        cfg = replace(cfg, fmt=fmt, scale_block=cfg.dstate)
+    T = 16
+    A, D = workloads.layer_params(cfg)
+    ins = [workloads.step_inputs(cfg, t) for t in range(1, T + 1)]
+    stack = lambda i: to_dev(np.stack([ins[t][i][None] for t in range(T)]))
+    xs, dts, Bs, Cs = (stack(i) for i in range(4))
+    sb = cfg.scale_block if oracle.has_block_scale(cfg.fmt) else 0
+
+    def run(overlap):
+        prev = ssdq.set_launch_overlap(overlap)
+        try:
+            st_h, sc_h = oracle.new_state(cfg.state_shape, cfg.fmt, sb)
+            st, sc = codes_to_dev(st_h, cfg.fmt), to_dev(sc_h)
+            desc = ssdq.make_desc(st, sc, cfg.fmt, A=to_dev(A), D=to_dev(D), rule=ssdq.WEYL,
+                                  weyl=ssdq.weyl_offsets_init(0, 0, cfg.weyl_block), scale_block=sb)
+            y = torch.zeros_like(xs)
+            ssdq.ssd_decode_run([desc], 1, T, ssdq.make_step_inputs(xs, dts, Bs, Cs, y))
+            torch.cuda.synchronize()
+            return st, sc, y
+        finally:
+            ssdq.set_launch_overlap(prev)
+
+    s0, c0, y0 = run(False)
+    for _ in range(3):
+        s1, c1, y1 = run(True)
+        assert torch.equal(s0, s1) and (c0 is None or torch.equal(c0, c1)) and torch.equal(y0, y1)
