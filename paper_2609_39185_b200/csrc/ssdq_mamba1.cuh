@@ -165,7 +165,7 @@ __global__ void __launch_bounds__(kThreads, RULE == RULE_RTN ? 8 : 6) ssd_update
         for (int c = 0; c < CH; ++c) unpack_lane<FMT>(raw[c], hin + c * EPL);
         f32x2 hn[N / 2];
         f32x2 dot2 = pack2(__fmul_rn(Dv, xv), 0.0f);
-        float amax = 0.0f;
+        [[maybe_unused]] float amax = 0.0f;
 #pragma unroll
         for (int i = 0; i < N / 4; ++i) {
             const float4 bb = Bp[i], cc = Cp[i];

@@ -86,7 +86,7 @@ __global__ void __launch_bounds__(kThreads, SSDQ_STREAM_MINB) ssd_update_stream_
 
     auto issue = [&](uint32_t stage) {
         // debug builds: the item's codes, x and scales must lie inside the caller's buffers (else nothing is copied)
-        const uint64_t frow = (uint64_t)(f_x - p.x);
+        [[maybe_unused]] const uint64_t frow = (uint64_t)(f_x - p.x);
         bool mem_ok = SSDQ_RANGE_OK(p, DBG_STATE, frow * LPR + lis, (RPS - 1) * LPR + 1, state_vecs) && SSDQ_RANGE_OK(p, DBG_ROWS, frow, RPS, rows) &&
                       SSDQ_RANGE_OK(p, DBG_SCALES, frow * SPR + (ROW_SCALE ? 0u : lis), (RPS - 1) * SPR + 1, scales);
         if (mem_ok) {
@@ -159,7 +159,7 @@ __global__ void __launch_bounds__(kThreads, SSDQ_STREAM_MINB) ssd_update_stream_
             A_next = __ldg(p.A + h_n);
             D_next = (p.D && lis == 0) ? __ldg(p.D + h_n) : 0.0f;
         }
-        const uint64_t crow = (uint64_t)(c_y - p.y) - lis / (LPR / 4);
+        [[maybe_unused]] const uint64_t crow = (uint64_t)(c_y - p.y) - lis / (LPR / 4);
         const bool mem_ok = SSDQ_RANGE_OK(p, DBG_STATE, crow * LPR + lis, (RPS - 1) * LPR + 1, state_vecs) && SSDQ_RANGE_OK(p, DBG_ROWS, crow, RPS, rows) &&
                             SSDQ_RANGE_OK(p, DBG_SCALES, crow * SPR + (ROW_SCALE ? 0u : lis), (RPS - 1) * SPR + 1, scales);
         uint32_t acc_row = 0;

@@ -51,7 +51,7 @@ __device__ __forceinline__ uint4 round_pack_lane(const float* v, uint32_t acc0, 
                                                  uint32_t g_hi, uint32_t step_t, uint32_t layer, uint32_t key0,
                                                  uint32_t key1, float qmax) {
     constexpr int EPL = Fmt<FMT>::kEpl;
-    uint32_t w[4];
+    uint32_t w[4] = {0u, 0u, 0u, 0u};       // (every path below sets all four; the one-byte formats return early)
     if constexpr (FMT == FMT_FP32) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) w[i] = __float_as_uint(v[i]);
