@@ -195,7 +195,7 @@ __global__ void __launch_bounds__(kThreads, RULE == RULE_RTN ? 8 : 6) ssd_update
         float v[N];
         if constexpr (Fmt<FMT>::kScaled) {
             const float s = fmaxf(__fdiv_rn(amax, p.scale_top), 1.17549435e-38f);
-            const float rinv = __frcp_rn(s);
+            const float rinv = rcp_scale(s);
             const f32x2 rinv2 = pack2(rinv, rinv);
 #pragma unroll
             for (int q = 0; q < N / 2; ++q) unpack2(mul2_rn(hn[q], rinv2), v[2 * q], v[2 * q + 1]);

@@ -206,7 +206,7 @@ __global__ void __launch_bounds__(kThreads, SSDQ_STREAM_MINB) ssd_update_stream_
                 for (int off = LPR / 2; off > 0; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, off));
             }
             const float s = fmaxf(div_by_top(amax, top, inv_top), 1.17549435e-38f);
-            const float rinv = __frcp_rn(s);
+            const float rinv = rcp_scale(s);
             const f32x2 rinv2 = pack2(rinv, rinv);
             float v[EPL];
 #pragma unroll
